@@ -1,0 +1,184 @@
+/*
+ * skipdecode.h - C ABI of the SkipDecode decode path for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the batched autoregressive decode step of an OPT-style
+ * decoder in which every token of the batch at one sequence position uses the
+ * same set of layers (Section 2.1 of the paper), the number of layers follows
+ * a monotonically non-increasing per-position budget between a maximum and a
+ * minimum (Sections 2.2 and 2.3), and the budget is spent on the top layers
+ * while the lower ones are bypassed, optionally after a few warm-up layers at
+ * the bottom (Section 2.4).  Because budgets never grow, keys and values that
+ * earlier positions wrote in the layers that still run are read as they are
+ * and never recomputed (Section 2.2).
+ *
+ * Conventions
+ *   - "host" / "device" in a comment says where a pointer must live.
+ *   - The caller owns every buffer: weights, the arena, token and logit
+ *     buffers, and the CUDA stream.  The library allocates no device memory;
+ *     it owns only the host-side handle.  Weight buffers are referenced, not
+ *     copied: they must stay valid until sd_destroy.
+ *   - Work is enqueued on the stream given to sd_create; calls return without
+ *     synchronising unless stated.  Device outputs are valid once the stream
+ *     reaches that point.
+ *   - Every function returns 0 (SD_OK) or a negative sd_error.  A call that
+ *     fails before enqueueing work changes no state.  Nothing aborts, throws
+ *     or traps on the device.
+ *   - Call order: sd_create -> sd_schedule -> sd_prefill -> sd_decode_step at
+ *     positions P, P+1, ..., P+gen_len-1.  A new sd_prefill starts a new batch
+ *     of sequences; sd_schedule may be called again between batches.
+ *   - Not thread-safe per handle.
+ */
+#ifndef SKIPDECODE_H
+#define SKIPDECODE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sd_handle sd_handle;
+
+typedef enum {
+  SD_OK = 0,
+  SD_ERR_ARG = -1,       /* NULL pointer, non-positive size, unsupported shape               */
+  SD_ERR_STATE = -2,     /* schedule or prefill missing                                        */
+  SD_ERR_POSITION = -3,  /* position out of order, past the schedule, or >= max_pos          */
+  SD_ERR_CAPACITY = -4,  /* arena too small, batch/prompt/generation beyond the configuration */
+  SD_ERR_CUDA = -5,      /* a CUDA call or launch failed                                      */
+  SD_ERR_DEVICE = -6     /* the device status word is non-zero (see sd_status)                */
+} sd_error;
+
+enum { SD_DTYPE_FP32 = 0, SD_DTYPE_BF16 = 1 };
+
+/* Model and limits.  Plain data, copied by sd_create.
+ * dtype selects the storage type of weights, GEMM input operands and the KV
+ * cache; the residual stream, LayerNorm statistics, softmax, accumulators and
+ * logits are fp32 in both modes.  head_dim = d_model / n_heads must be 32, 64
+ * or 128; d_model and d_ffn must be multiples of 8; max_prompt + max_gen <= max_pos. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, d_ffn, vocab, max_pos;
+  int32_t max_batch, max_prompt, max_gen;
+  int32_t dtype;      /* SD_DTYPE_FP32 or SD_DTYPE_BF16 */
+  float ln_eps;       /* 1e-5 for OPT */
+} sd_config;
+
+/* DEVICE pointers to the weights, each matrix row-major [out, in] as a linear
+ * layer stores it, element type per sd_config.dtype, 16-byte aligned.  The
+ * per-layer members are HOST arrays of n_layers device pointers.  lm_head may
+ * be NULL: the head is then tied to tok_emb (OPT's default). */
+typedef struct {
+  const void *tok_emb, *pos_emb;              /* [vocab, d], [max_pos, d]                 */
+  const void *const *ln1_g, *const *ln1_b;    /* [d] each                                 */
+  const void *const *w_qkv, *const *b_qkv;    /* [3d, d] rows ordered q, k, v ; [3d]      */
+  const void *const *w_o, *const *b_o;        /* [d, d] ; [d]                             */
+  const void *const *ln2_g, *const *ln2_b;    /* [d] each                                 */
+  const void *const *w_fc1, *const *b_fc1;    /* [d_ffn, d] ; [d_ffn]                     */
+  const void *const *w_fc2, *const *b_fc2;    /* [d, d_ffn] ; [d]                         */
+  const void *lnf_g, *lnf_b, *lm_head;        /* [d], [d], [vocab, d] or NULL             */
+} sd_weights;
+
+/* Cache sizing plan.  Each layer's KV cache holds max_prompt positions plus
+ * one position for every generated index at which the schedule
+ * (max_layers, min_layers, warmup, gen_len) runs that layer: a layer that has
+ * dropped out of a monotone schedule is never appended to again (Section 2.2).
+ * full_capacity = 1 sizes every layer for max_prompt + max_gen positions so
+ * that any schedule, including the all-layers baseline, fits. */
+typedef struct {
+  int32_t max_layers, min_layers, warmup, gen_len, full_capacity;
+} sd_plan;
+
+/* Bytes of device memory the arena must provide for (config, plan).
+ * out: host.  Errors: SD_ERR_ARG. */
+int sd_arena_bytes(const sd_config *cfg, const sd_plan *plan, size_t *out);
+
+/* Creates a handle.  arena: device, 256-byte aligned, arena_bytes >= sd_arena_bytes;
+ * it holds the per-layer KV caches [max_batch, n_heads, capacity_l, head_dim] for K
+ * and for V, the activation buffers, the split-KV partial results and a status word.
+ * stream: a cudaStream_t (NULL = the legacy default stream).  The arena's status and
+ * counters are cleared on the stream.
+ * Errors: SD_ERR_ARG (shape rules above, NULL weights), SD_ERR_CAPACITY (arena too
+ * small), SD_ERR_CUDA. */
+int sd_create(const sd_config *cfg, const sd_weights *weights, const sd_plan *plan,
+              void *arena, size_t arena_bytes, void *stream, sd_handle **out);
+
+/* Computes and installs the per-position layer budget (Section 2.3): generated
+ * index g = position - prompt_len in [0, gen_len) gets
+ *     n_active[g] = round_half_up((1 - t) * max_layers + t * min_layers),  t = g / (gen_len - 1)
+ * (n_active[0] = max_layers when gen_len = 1), computed in integers, so the first
+ * generated position gets max_layers and the last min_layers.  The layers that run
+ * at g are [0, warmup) and [top_begin[g], n_layers), top_begin[g] = n_layers -
+ * (n_active[g] - warmup) (Section 2.4); prompt positions use every layer.
+ * n_active, top_begin: host, gen_len int32 each, either may be NULL.
+ * Requires 0 <= warmup < min_layers <= max_layers <= n_layers, 1 <= gen_len <= max_gen.
+ * Errors: SD_ERR_ARG; SD_ERR_CAPACITY if a layer would need more cache positions
+ * than the plan given to sd_create reserved.  Resets the sequence state. */
+int sd_schedule(sd_handle *h, int max_layers, int min_layers, int warmup, int gen_len,
+                int32_t *n_active, int32_t *top_begin);
+
+/* The same arithmetic as sd_schedule without a handle or a device (host only):
+ * fills n_active[gen_len] and top_begin[gen_len] for a model of n_layers layers.
+ * Errors: SD_ERR_ARG. */
+int sd_schedule_compute(int n_layers, int max_layers, int min_layers, int warmup, int gen_len,
+                        int32_t *n_active, int32_t *top_begin);
+
+/* Cache positions the plan reserves per layer (host only): capacity[n_layers]. */
+int sd_layer_capacity(const sd_config *cfg, const sd_plan *plan, int32_t *capacity);
+
+/* Processes the prompt with all layers (Section 2.3): fills cache positions
+ * 0..P-1 of every layer and writes the logits of position P-1.
+ * d_tokens: device int32 [B, P] row-major, ids in [0, vocab).  d_logits: device
+ * fp32 [B, vocab].  1 <= B <= max_batch, 1 <= P <= max_prompt, P + gen_len <= max_pos.
+ * Errors: SD_ERR_ARG, SD_ERR_STATE (no schedule), SD_ERR_CAPACITY, SD_ERR_CUDA. */
+int sd_prefill(sd_handle *h, const int32_t *d_tokens, int B, int P, float *d_logits);
+
+/* One decode step (Sections 2.1-2.4): the B tokens at `position` run through the
+ * layers the schedule makes active there, append their keys/values in those
+ * layers only, attend to cache positions 0..position, and produce next-token
+ * logits.  d_token_ids: device int32 [B]; d_logits: device fp32 [B, vocab].
+ * position must be P + (number of decode steps since sd_prefill).
+ * Errors: SD_ERR_ARG, SD_ERR_STATE (no prefill), SD_ERR_POSITION, SD_ERR_CUDA. */
+int sd_decode_step(sd_handle *h, const int32_t *d_token_ids, int position, float *d_logits);
+
+/* The same step with HOST buffers: copies h_token_ids [B] to the device, runs the
+ * step, copies the logits [B, vocab] back and synchronises the stream.  Pinned
+ * host memory makes the copies asynchronous to the host but is not required. */
+int sd_decode_step_host(sd_handle *h, const int32_t *h_token_ids, int position, float *h_logits);
+
+/* Greedy choice: d_next[b] = lowest index attaining the maximum of d_logits[b, :].
+ * d_logits: device fp32 [B, vocab]; d_next: device int32 [B]. */
+int sd_greedy(sd_handle *h, const float *d_logits, int B, int32_t *d_next);
+
+/* Synchronises the stream and reads the device status word (0 = no error; kernels
+ * set bits on an out-of-range token id or a bounded wait that expired).
+ * Returns SD_ERR_DEVICE when it is non-zero. */
+int sd_status(sd_handle *h, int32_t *device_status);
+
+/* Decode steps run since sd_create and the number of layer executions they made
+ * (their ratio is the mean active layers per generated token). */
+int sd_stats(sd_handle *h, int64_t *steps, int64_t *layer_steps);
+
+/* Tuning knobs; every value of every option computes the same function. */
+enum {
+  SD_OPT_GRAPHS = 1,       /* 1 (default): replay one CUDA graph per step shape; 0: plain launches */
+  SD_OPT_ATTN_CHUNK = 2,   /* keys per split of the decode attention (multiple of 32); 0 = automatic */
+  SD_OPT_GEMM = 3,         /* 0 = automatic; 1 = CUDA-core GEMMs only (bf16 mode as well)          */
+  SD_OPT_TIMING = 4        /* 1: record per-kernel-class device time (plain launches, slower)      */
+};
+int sd_set_option(sd_handle *h, int option, int value);
+
+/* Device time and launch count accumulated per kernel class while SD_OPT_TIMING is
+ * on; synchronises the stream.  ms, launches: host. */
+enum { SD_K_EMBED = 0, SD_K_LAYERNORM = 1, SD_K_GEMM = 2, SD_K_KV_APPEND = 3,
+       SD_K_ATTENTION = 4, SD_K_COMBINE = 5, SD_K_LM_HEAD = 6, SD_K_COUNT = 7 };
+int sd_kernel_time(sd_handle *h, int kernel_class, double *ms, int64_t *launches);
+int sd_kernel_time_reset(sd_handle *h);
+
+const char *sd_strerror(int code);
+void sd_destroy(sd_handle *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SKIPDECODE_H */
