@@ -1,0 +1,563 @@
+// Host side of the C ABI declared in include/skipdecode.h: argument checks, the
+// integer schedule, arena carving, and the launch sequence of one prefill / one
+// decode step (replayed from a CUDA graph per step shape when enabled).
+#include "../../include/skipdecode.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <tuple>
+#include <type_traits>
+#include <vector>
+
+#include "kernels.cuh"
+#include "gemm_tc.cuh"
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+constexpr size_t kAlign = 256;
+constexpr int kPrefillTokens = 4096;   // query rows per prefill pass (whole batch rows)
+constexpr int kMinChunk = 32;          // smallest split of the decode attention, in keys
+
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Arena {            // byte offsets into the caller's arena
+  std::vector<size_t> k_off, v_off;
+  std::vector<int> cap;
+  size_t x, u, qkv, o, y, part_acc, part_ml, row_index, ids, logits, scalars, total;
+  int rows_max;
+  size_t part_slots;
+};
+
+struct Timed { cudaEvent_t a, b; int cls; };
+
+}  // namespace
+
+struct sd_handle {
+  sd_config cfg;
+  sd_plan plan;
+  int hd, esize;
+  std::vector<const void*> ln1_g, ln1_b, w_qkv, b_qkv, w_o, b_o, ln2_g, ln2_b, w_fc1, b_fc1, w_fc2, b_fc2;
+  const void *tok_emb, *pos_emb, *lnf_g, *lnf_b, *lm_head;
+  char* arena;
+  Arena A;
+  cudaStream_t stream;
+  // schedule / sequence state
+  std::vector<int> n_active, top_begin;
+  int warmup = 0, gen_len = 0;
+  bool have_schedule = false, have_prefill = false;
+  int B = 0, P = 0, next_pos = 0;
+  int64_t steps = 0, layer_steps = 0;
+  // options
+  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0;
+  // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
+  std::map<std::tuple<int, int, int, int, int, const void*, const void*>, cudaGraphExec_t> graphs;
+  // timing
+  std::vector<Timed> timed;
+  double k_ms[SD_K_COUNT] = {};
+  int64_t k_launches[SD_K_COUNT] = {};
+  sd::TcContext tc;
+
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(arena + off); }
+  int* status() const { return at<int>(A.scalars); }
+  int* d_pos() const { return at<int>(A.scalars) + 1; }
+};
+
+namespace {
+
+bool valid_config(const sd_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->d_ffn < 8 || c->vocab < 1 || c->max_pos < 1) return false;
+  if (c->max_batch < 1 || c->max_prompt < 1 || c->max_gen < 1) return false;
+  if (c->dtype != SD_DTYPE_FP32 && c->dtype != SD_DTYPE_BF16) return false;
+  if (c->d_model % c->n_heads) return false;
+  const int hd = c->d_model / c->n_heads;
+  if (hd != 32 && hd != 64 && hd != 128) return false;
+  if (c->d_model % 8 || c->d_ffn % 8) return false;
+  if (!(c->ln_eps > 0.f)) return false;
+  if ((int64_t)c->max_prompt + c->max_gen > c->max_pos) return false;
+  return true;
+}
+
+bool valid_schedule_args(int n_layers, int mx, int mn, int w, int G) {
+  return 0 <= w && w < mn && mn <= mx && mx <= n_layers && G >= 1;
+}
+
+// Section 2.3: the line (1 - t) max + t min with t = g / (G - 1), rounded to nearest with
+// halves up, in integers: min + floor((2 (G-1-g) (max-min) + (G-1)) / (2 (G-1))).
+int budget_at(int mx, int mn, int g, int G) {
+  if (G == 1) return mx;
+  const int64_t den = G - 1, D = mx - mn;
+  return mn + (int)((2 * (den - g) * D + den) / (2 * den));
+}
+
+// number of generated indices at which layer l runs under (mx, mn, w, G)
+void layer_counts(int L, int mx, int mn, int w, int G, std::vector<int>& count) {
+  count.assign(L, 0);
+  for (int g = 0; g < G; ++g) {
+    const int n = budget_at(mx, mn, g, G), top = L - (n - w);
+    for (int l = 0; l < L; ++l)
+      if (l < w || l >= top) ++count[l];
+  }
+}
+
+bool valid_plan(const sd_config* c, const sd_plan* p) {
+  return p && valid_schedule_args(c->n_layers, p->max_layers, p->min_layers, p->warmup, p->gen_len) &&
+         p->gen_len <= c->max_gen;
+}
+
+void carve(const sd_config& c, const sd_plan& p, Arena& A) {
+  const int L = c.n_layers, d = c.d_model, H = c.n_heads, hd = d / H;
+  const size_t e = c.dtype == SD_DTYPE_FP32 ? 4 : 2;
+  std::vector<int> count;
+  layer_counts(L, p.max_layers, p.min_layers, p.warmup, p.gen_len, count);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  A.k_off.resize(L); A.v_off.resize(L); A.cap.resize(L);
+  for (int l = 0; l < L; ++l) {
+    A.cap[l] = c.max_prompt + (p.full_capacity ? c.max_gen : count[l]);
+    const size_t bytes = (size_t)c.max_batch * H * A.cap[l] * hd * e;
+    A.k_off[l] = take(bytes);
+    A.v_off[l] = take(bytes);
+  }
+  const int chunk_rows = std::max(1, kPrefillTokens / c.max_prompt) * c.max_prompt;
+  A.rows_max = std::max(c.max_batch, chunk_rows);
+  const size_t R = A.rows_max;
+  A.x = take(R * d * 4);
+  A.u = take(R * d * e);
+  A.qkv = take(R * 3 * d * 4);
+  A.o = take(R * d * e);
+  A.y = take(R * (size_t)c.d_ffn * e);
+  const int maxT = c.max_prompt + c.max_gen;
+  A.part_slots = std::max((size_t)c.max_batch * H * ((maxT + kMinChunk - 1) / kMinChunk), R * H);
+  A.part_acc = take(A.part_slots * hd * 4);
+  A.part_ml = take(A.part_slots * 2 * 4);
+  A.row_index = take((size_t)c.max_batch * 4);
+  A.ids = take((size_t)c.max_batch * 4);
+  A.logits = take((size_t)c.max_batch * c.vocab * 4);
+  A.scalars = take(256);
+  A.total = off;
+}
+
+__global__ void set_int_kernel(int* p, int v) { *p = v; }
+__global__ void last_rows_kernel(int* idx, int n, int P) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) idx[i] = i * P + P - 1;
+}
+
+// ---- launch helpers -------------------------------------------------------------------
+
+struct Launcher {
+  sd_handle* h;
+  bool timing;
+  int err = 0;
+  void begin(int cls) {
+    if (!timing) return;
+    Timed t; t.cls = cls;
+    cudaEventCreate(&t.a); cudaEventCreate(&t.b);
+    cudaEventRecord(t.a, h->stream);
+    h->timed.push_back(t);
+  }
+  void end() {
+    if (cudaGetLastError() != cudaSuccess) err = SD_ERR_CUDA;
+    if (timing) cudaEventRecord(h->timed.back().b, h->stream);
+  }
+};
+
+template <typename T>
+void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, const T* bias, int M, int N, int K,
+                 void* out, int ldo, int epi) {
+  sd_handle* h = Lc.h;
+  Lc.begin(cls);
+  bool done = false;
+  if (std::is_same<T, bf16>::value && h->opt_gemm != 1)
+    done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status());
+  if (!done) {
+    dim3 grid((N + 63) / 64, (M + 63) / 64);
+    if (epi == sd::EPI_STORE_F32)
+      sd::gemm_simt_kernel<T, sd::EPI_STORE_F32><<<grid, 256, 0, h->stream>>>(A, K, W, K, bias, M, N, K, out, ldo);
+    else if (epi == sd::EPI_RELU_T)
+      sd::gemm_simt_kernel<T, sd::EPI_RELU_T><<<grid, 256, 0, h->stream>>>(A, K, W, K, bias, M, N, K, out, ldo);
+    else
+      sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32><<<grid, 256, 0, h->stream>>>(A, K, W, K, bias, M, N, K, out, ldo);
+  }
+  Lc.end();
+}
+
+template <typename T, int HD>
+void launch_attention_hd(Launcher& Lc, const T* Kc, const T* Vc, int cap, int rows, sd::RowMap map, int chunk,
+                         int n_chunks) {
+  sd_handle* h = Lc.h;
+  const int H = h->cfg.n_heads;
+  Lc.begin(SD_K_ATTENTION);
+  dim3 grid(rows * H, n_chunks);
+  sd::attn_partial_kernel<T, HD, 4><<<grid, 128, 0, h->stream>>>(
+      h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks,
+      h->at<float>(h->A.part_acc), h->at<float>(h->A.part_ml));
+  Lc.end();
+  Lc.begin(SD_K_COMBINE);
+  sd::attn_combine_kernel<T, HD><<<rows * H, HD < 64 ? 32 : 64, 0, h->stream>>>(
+      h->at<float>(h->A.part_acc), h->at<float>(h->A.part_ml), h->at<T>(h->A.o), H, cap, map, chunk, n_chunks);
+  Lc.end();
+}
+
+template <typename T>
+void launch_attention(Launcher& Lc, const T* Kc, const T* Vc, int cap, int rows, sd::RowMap map, int chunk, int n_chunks) {
+  switch (Lc.h->hd) {
+    case 32: launch_attention_hd<T, 32>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks); break;
+    case 64: launch_attention_hd<T, 64>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks); break;
+    default: launch_attention_hd<T, 128>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks); break;
+  }
+}
+
+int ln_threads(int d) { return std::max(32, std::min(256, (d / 4 + 31) / 32 * 32)); }
+
+// One decoder layer over `rows` query rows (Sections 2.1, 2.2): LN1 -> QKV -> append K,V at
+// the rows' positions -> attention over cache positions 0..pos -> out-proj (+residual) ->
+// LN2 -> fc1 + ReLU -> fc2 (+residual).
+template <typename T>
+void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int n_chunks) {
+  sd_handle* h = Lc.h;
+  const sd_config& c = h->cfg;
+  const int d = c.d_model, f = c.d_ffn;
+  float* x = h->at<float>(h->A.x);
+  T* u = h->at<T>(h->A.u);
+  float* qkv = h->at<float>(h->A.qkv);
+  T* o = h->at<T>(h->A.o);
+  T* y = h->at<T>(h->A.y);
+  T* Kc = h->at<T>(h->A.k_off[l]);
+  T* Vc = h->at<T>(h->A.v_off[l]);
+  const int cap = h->A.cap[l];
+
+  Lc.begin(SD_K_LAYERNORM);
+  sd::layernorm_kernel<T><<<rows, ln_threads(d), 0, h->stream>>>(x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
+  Lc.end();
+  launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
+  Lc.begin(SD_K_KV_APPEND);
+  sd::kv_append_kernel<T><<<rows, 256, 0, h->stream>>>(qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
+  Lc.end();
+  launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
+  launch_gemm<T>(Lc, SD_K_GEMM, o, (const T*)h->w_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
+  Lc.begin(SD_K_LAYERNORM);
+  sd::layernorm_kernel<T><<<rows, ln_threads(d), 0, h->stream>>>(x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
+  Lc.end();
+  launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f, sd::EPI_RELU_T);
+  launch_gemm<T>(Lc, SD_K_GEMM, y, (const T*)h->w_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
+}
+
+template <typename T>
+void enqueue_embed(Launcher& Lc, const int32_t* ids, int rows, sd::RowMap map) {
+  sd_handle* h = Lc.h;
+  Lc.begin(SD_K_EMBED);
+  sd::embed_pos_kernel<T><<<rows, 256, 0, h->stream>>>(ids, (const T*)h->tok_emb, (const T*)h->pos_emb, h->at<float>(h->A.x),
+                                                      h->cfg.d_model, h->cfg.vocab, h->cfg.max_pos, map, h->status());
+  Lc.end();
+}
+
+// final LayerNorm of `rows` rows (gathered through row_index when given) and the LM head
+template <typename T>
+void enqueue_head(Launcher& Lc, int rows, const int* row_index, float* d_logits) {
+  sd_handle* h = Lc.h;
+  const sd_config& c = h->cfg;
+  Lc.begin(SD_K_LAYERNORM);
+  sd::layernorm_kernel<T><<<rows, ln_threads(c.d_model), 0, h->stream>>>(h->at<float>(h->A.x), (const T*)h->lnf_g, (const T*)h->lnf_b,
+                                                                        h->at<T>(h->A.u), c.d_model, c.ln_eps, row_index);
+  Lc.end();
+  launch_gemm<T>(Lc, SD_K_LM_HEAD, h->at<T>(h->A.u), (const T*)h->lm_head, (const T*)nullptr, rows, c.vocab, c.d_model,
+                 d_logits, c.vocab, sd::EPI_STORE_F32);
+}
+
+// keys per split for a decode step with `rows` x H query-heads and T keys each
+int pick_chunk(const sd_handle* h, int rows, int T) {
+  if (h->opt_chunk > 0) return h->opt_chunk;
+  const long rh = (long)rows * h->cfg.n_heads;
+  const long want = 8L * 148;                       // blocks in flight to cover the SMs
+  for (int chunk : {512, 256, 128, 64}) {
+    if (rh * ((T + chunk - 1) / chunk) >= want) return chunk;
+  }
+  return kMinChunk;
+}
+
+template <typename T>
+int enqueue_decode(sd_handle* h, const int32_t* d_ids, int pos, bool pos_from_device, float* d_logits, int n, int chunk,
+                   int n_chunks, bool timing) {
+  Launcher Lc{h, timing};
+  const int L = h->cfg.n_layers, w = h->warmup, top = L - (n - w);
+  sd::RowMap map{1, 0, pos, pos_from_device ? h->d_pos() : nullptr};
+  enqueue_embed<T>(Lc, d_ids, h->B, map);
+  for (int l = 0; l < L; ++l) {
+    if (!(l < w || l >= top)) continue;             // bypassed layer: identity, no K/V written (Section 2.4)
+    enqueue_layer<T>(Lc, l, h->B, map, chunk, n_chunks);
+  }
+  enqueue_head<T>(Lc, h->B, nullptr, d_logits);
+  return Lc.err;
+}
+
+template <typename T>
+int run_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_logits) {
+  Launcher Lc{h, h->opt_timing != 0};
+  const int L = h->cfg.n_layers;
+  const int per = std::max(1, kPrefillTokens / P);
+  for (int b0 = 0; b0 < B; b0 += per) {
+    const int nb = std::min(per, B - b0), rows = nb * P;
+    sd::RowMap map{P, b0, 0, nullptr};
+    enqueue_embed<T>(Lc, d_tokens + (size_t)b0 * P, rows, map);
+    const int chunk = (P + kMinChunk - 1) / kMinChunk * kMinChunk;   // one split: every row reads keys 0..pos
+    for (int l = 0; l < L; ++l) enqueue_layer<T>(Lc, l, rows, map, chunk, 1);
+    last_rows_kernel<<<(nb + 127) / 128, 128, 0, h->stream>>>(h->at<int>(h->A.row_index), nb, P);
+    enqueue_head<T>(Lc, nb, h->at<int>(h->A.row_index), d_logits + (size_t)b0 * h->cfg.vocab);
+  }
+  return Lc.err;
+}
+
+void collect_timing(sd_handle* h) {
+  if (h->timed.empty()) return;
+  cudaStreamSynchronize(h->stream);
+  for (Timed& t : h->timed) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, t.a, t.b) == cudaSuccess) { h->k_ms[t.cls] += ms; h->k_launches[t.cls] += 1; }
+    cudaEventDestroy(t.a); cudaEventDestroy(t.b);
+  }
+  h->timed.clear();
+}
+
+void drop_graphs(sd_handle* h) {
+  for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+  h->graphs.clear();
+}
+
+int decode_step_impl(sd_handle* h, const int32_t* d_ids, int position, float* d_logits) {
+  if (!h || !d_ids || !d_logits) return SD_ERR_ARG;
+  if (!h->have_schedule || !h->have_prefill) return SD_ERR_STATE;
+  const int g = position - h->P;
+  if (position != h->next_pos || g < 0 || g >= h->gen_len || position >= h->cfg.max_pos) return SD_ERR_POSITION;
+  const int n = h->n_active[g];
+  const int T = position + 1;
+  const int chunk = pick_chunk(h, h->B, T);
+  const int n_chunks = (T + chunk - 1) / chunk;
+  const bool bf = h->cfg.dtype == SD_DTYPE_BF16;
+  int err = 0;
+  const bool graphs = h->opt_graphs && !h->opt_timing && h->stream != nullptr;
+  if (!graphs) {
+    err = bf ? enqueue_decode<bf16>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0)
+             : enqueue_decode<float>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0);
+  } else {
+    auto key = std::make_tuple(h->B, n, h->warmup, chunk, n_chunks, (const void*)d_ids, (const void*)d_logits);
+    auto it = h->graphs.find(key);
+    if (it == h->graphs.end()) {
+      if (h->graphs.size() >= 256) drop_graphs(h);
+      cudaGraph_t graph = nullptr;
+      if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+      err = bf ? enqueue_decode<bf16>(h, d_ids, position, true, d_logits, n, chunk, n_chunks, false)
+               : enqueue_decode<float>(h, d_ids, position, true, d_logits, n, chunk, n_chunks, false);
+      const cudaError_t ce = cudaStreamEndCapture(h->stream, &graph);
+      if (ce != cudaSuccess || err || !graph) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return SD_ERR_CUDA; }
+      cudaGraphExec_t exec = nullptr;
+      const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (ie != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+      it = h->graphs.emplace(key, exec).first;
+    }
+    set_int_kernel<<<1, 1, 0, h->stream>>>(h->d_pos(), position);
+    if (cudaGraphLaunch(it->second, h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  }
+  if (err) return err;
+  h->next_pos = position + 1;
+  h->steps += 1;
+  h->layer_steps += n;
+  return SD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sd_arena_bytes(const sd_config* cfg, const sd_plan* plan, size_t* out) {
+  if (!valid_config(cfg) || !out || !valid_plan(cfg, plan)) return SD_ERR_ARG;
+  Arena A;
+  carve(*cfg, *plan, A);
+  *out = A.total;
+  return SD_OK;
+}
+
+int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, void* arena, size_t arena_bytes,
+              void* stream, sd_handle** out) {
+  if (!valid_config(cfg) || !w || !out || !arena || !valid_plan(cfg, plan)) return SD_ERR_ARG;
+  if (reinterpret_cast<uintptr_t>(arena) % kAlign) return SD_ERR_ARG;
+  const int L = cfg->n_layers;
+  const void* const* per_layer[] = {w->ln1_g, w->ln1_b, w->w_qkv, w->b_qkv, w->w_o, w->b_o,
+                                    w->ln2_g, w->ln2_b, w->w_fc1, w->b_fc1, w->w_fc2, w->b_fc2};
+  for (auto arr : per_layer) {
+    if (!arr) return SD_ERR_ARG;
+    for (int l = 0; l < L; ++l)
+      if (!arr[l]) return SD_ERR_ARG;
+  }
+  if (!w->tok_emb || !w->pos_emb || !w->lnf_g || !w->lnf_b) return SD_ERR_ARG;
+  sd_handle* h = new (std::nothrow) sd_handle();
+  if (!h) return SD_ERR_ARG;
+  h->cfg = *cfg;
+  h->plan = *plan;
+  h->hd = cfg->d_model / cfg->n_heads;
+  h->esize = cfg->dtype == SD_DTYPE_FP32 ? 4 : 2;
+  carve(*cfg, *plan, h->A);
+  if (h->A.total > arena_bytes) { delete h; return SD_ERR_CAPACITY; }
+  auto copy = [&](std::vector<const void*>& dst, const void* const* src) { dst.assign(src, src + L); };
+  copy(h->ln1_g, w->ln1_g); copy(h->ln1_b, w->ln1_b); copy(h->w_qkv, w->w_qkv); copy(h->b_qkv, w->b_qkv);
+  copy(h->w_o, w->w_o); copy(h->b_o, w->b_o); copy(h->ln2_g, w->ln2_g); copy(h->ln2_b, w->ln2_b);
+  copy(h->w_fc1, w->w_fc1); copy(h->b_fc1, w->b_fc1); copy(h->w_fc2, w->w_fc2); copy(h->b_fc2, w->b_fc2);
+  h->tok_emb = w->tok_emb; h->pos_emb = w->pos_emb; h->lnf_g = w->lnf_g; h->lnf_b = w->lnf_b;
+  h->lm_head = w->lm_head ? w->lm_head : w->tok_emb;
+  h->arena = static_cast<char*>(arena);
+  h->stream = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(h->arena + h->A.scalars, 0, 256, h->stream) != cudaSuccess) { cudaGetLastError(); delete h; return SD_ERR_CUDA; }
+  sd::tc_init(h->tc);
+  *out = h;
+  return SD_OK;
+}
+
+int sd_schedule(sd_handle* h, int mx, int mn, int w, int G, int32_t* n_active, int32_t* top_begin) {
+  if (!h || !valid_schedule_args(h->cfg.n_layers, mx, mn, w, G) || G > h->cfg.max_gen) return SD_ERR_ARG;
+  const int L = h->cfg.n_layers;
+  std::vector<int> count;
+  layer_counts(L, mx, mn, w, G, count);
+  for (int l = 0; l < L; ++l)
+    if (h->cfg.max_prompt + count[l] > h->A.cap[l]) return SD_ERR_CAPACITY;
+  h->n_active.resize(G); h->top_begin.resize(G);
+  for (int g = 0; g < G; ++g) {
+    h->n_active[g] = budget_at(mx, mn, g, G);
+    h->top_begin[g] = L - (h->n_active[g] - w);
+    if (n_active) n_active[g] = h->n_active[g];
+    if (top_begin) top_begin[g] = h->top_begin[g];
+  }
+  h->warmup = w; h->gen_len = G;
+  h->have_schedule = true; h->have_prefill = false;
+  return SD_OK;
+}
+
+int sd_schedule_compute(int n_layers, int mx, int mn, int w, int G, int32_t* n_active, int32_t* top_begin) {
+  if (!valid_schedule_args(n_layers, mx, mn, w, G)) return SD_ERR_ARG;
+  for (int g = 0; g < G; ++g) {
+    const int n = budget_at(mx, mn, g, G);
+    if (n_active) n_active[g] = n;
+    if (top_begin) top_begin[g] = n_layers - (n - w);
+  }
+  return SD_OK;
+}
+
+int sd_layer_capacity(const sd_config* cfg, const sd_plan* plan, int32_t* capacity) {
+  if (!valid_config(cfg) || !valid_plan(cfg, plan) || !capacity) return SD_ERR_ARG;
+  Arena A;
+  carve(*cfg, *plan, A);
+  for (int l = 0; l < cfg->n_layers; ++l) capacity[l] = A.cap[l];
+  return SD_OK;
+}
+
+int sd_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_logits) {
+  if (!h || !d_tokens || !d_logits || B < 1 || P < 1) return SD_ERR_ARG;
+  if (!h->have_schedule) return SD_ERR_STATE;
+  if (B > h->cfg.max_batch || P > h->cfg.max_prompt || (int64_t)P + h->gen_len > h->cfg.max_pos) return SD_ERR_CAPACITY;
+  const int err = h->cfg.dtype == SD_DTYPE_BF16 ? run_prefill<bf16>(h, d_tokens, B, P, d_logits)
+                                                : run_prefill<float>(h, d_tokens, B, P, d_logits);
+  if (err) return err;
+  h->B = B; h->P = P; h->next_pos = P; h->have_prefill = true;
+  return SD_OK;
+}
+
+int sd_decode_step(sd_handle* h, const int32_t* d_token_ids, int position, float* d_logits) {
+  return decode_step_impl(h, d_token_ids, position, d_logits);
+}
+
+int sd_decode_step_host(sd_handle* h, const int32_t* h_ids, int position, float* h_logits) {
+  if (!h || !h_ids || !h_logits) return SD_ERR_ARG;
+  if (!h->have_schedule || !h->have_prefill) return SD_ERR_STATE;
+  int32_t* d_ids = h->at<int32_t>(h->A.ids);
+  float* d_logits = h->at<float>(h->A.logits);
+  if (cudaMemcpyAsync(d_ids, h_ids, (size_t)h->B * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  const int err = decode_step_impl(h, d_ids, position, d_logits);
+  if (err) return err;
+  if (cudaMemcpyAsync(h_logits, d_logits, (size_t)h->B * h->cfg.vocab * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  return SD_OK;
+}
+
+int sd_greedy(sd_handle* h, const float* d_logits, int B, int32_t* d_next) {
+  if (!h || !d_logits || !d_next || B < 1) return SD_ERR_ARG;
+  sd::greedy_kernel<<<B, 1024, 0, h->stream>>>(d_logits, h->cfg.vocab, d_next);
+  return cudaGetLastError() == cudaSuccess ? SD_OK : SD_ERR_CUDA;
+}
+
+int sd_status(sd_handle* h, int32_t* device_status) {
+  if (!h) return SD_ERR_ARG;
+  int32_t v = 0;
+  if (cudaMemcpyAsync(&v, h->status(), 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  if (device_status) *device_status = v;
+  return v ? SD_ERR_DEVICE : SD_OK;
+}
+
+int sd_stats(sd_handle* h, int64_t* steps, int64_t* layer_steps) {
+  if (!h) return SD_ERR_ARG;
+  if (steps) *steps = h->steps;
+  if (layer_steps) *layer_steps = h->layer_steps;
+  return SD_OK;
+}
+
+int sd_set_option(sd_handle* h, int option, int value) {
+  if (!h) return SD_ERR_ARG;
+  switch (option) {
+    case SD_OPT_GRAPHS: h->opt_graphs = value ? 1 : 0; return SD_OK;
+    case SD_OPT_ATTN_CHUNK:
+      if (value != 0 && (value < kMinChunk || value % kMinChunk)) return SD_ERR_ARG;
+      h->opt_chunk = value; return SD_OK;
+    case SD_OPT_GEMM:
+      if (value < 0 || value > 1) return SD_ERR_ARG;
+      if (value != h->opt_gemm) drop_graphs(h);
+      h->opt_gemm = value; return SD_OK;
+    case SD_OPT_TIMING:
+      if (h->opt_timing && !value) collect_timing(h);
+      h->opt_timing = value ? 1 : 0; return SD_OK;
+    default: return SD_ERR_ARG;
+  }
+}
+
+int sd_kernel_time(sd_handle* h, int cls, double* ms, int64_t* launches) {
+  if (!h || cls < 0 || cls >= SD_K_COUNT) return SD_ERR_ARG;
+  collect_timing(h);
+  if (ms) *ms = h->k_ms[cls];
+  if (launches) *launches = h->k_launches[cls];
+  return SD_OK;
+}
+
+int sd_kernel_time_reset(sd_handle* h) {
+  if (!h) return SD_ERR_ARG;
+  collect_timing(h);
+  for (int i = 0; i < SD_K_COUNT; ++i) { h->k_ms[i] = 0; h->k_launches[i] = 0; }
+  return SD_OK;
+}
+
+const char* sd_strerror(int code) {
+  switch (code) {
+    case SD_OK: return "ok";
+    case SD_ERR_ARG: return "invalid argument";
+    case SD_ERR_STATE: return "schedule or prefill missing";
+    case SD_ERR_POSITION: return "position out of order or outside the schedule";
+    case SD_ERR_CAPACITY: return "capacity exceeded";
+    case SD_ERR_CUDA: return "CUDA call failed";
+    case SD_ERR_DEVICE: return "device status word is set";
+    default: return "unknown error";
+  }
+}
+
+void sd_destroy(sd_handle* h) {
+  if (!h) return;
+  collect_timing(h);
+  drop_graphs(h);
+  sd::tc_destroy(h->tc);
+  delete h;
+}
+
+}  // extern "C"
