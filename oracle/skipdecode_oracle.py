@@ -167,14 +167,14 @@ def _causal_layer(h: torch.Tensor, lw: dict, n_heads: int, dtype) -> torch.Tenso
 # --------------------------------------------------------------------------- definition
 
 def forward_sequence(weights: dict, n_heads: int, tokens: torch.Tensor, active: torch.Tensor,
-                     dtype=torch.float64, return_hidden: bool = False):
+                     dtype=torch.float64, return_hidden: bool = False, logits_from: int = 0):
     """Logits at every position of tokens[B,S] under per-position layer sets.
 
     active[i, l] says whether layer l runs at position i.  A layer that does not
     run at a position is the identity there and contributes no key/value
     [Section 2.4]; the positions where a layer runs must form a prefix 0..m-1
     (monotone budgets, Section 2.2), otherwise a needed key would not exist and
-    the call raises.
+    the call raises.  Logits are returned for positions logits_from..S-1 only.
     """
     B, S = tokens.shape
     L = len(weights["layers"])
@@ -187,7 +187,7 @@ def forward_sequence(weights: dict, n_heads: int, tokens: torch.Tensor, active: 
         if m == 0:
             continue
         h = torch.cat([_causal_layer(h[:, :m], weights["layers"][l], n_heads, dtype), h[:, m:]], dim=1)
-    logits = _head(weights, h, dtype)
+    logits = _head(weights, h[:, logits_from:], dtype)
     return (logits, h) if return_hidden else logits
 
 

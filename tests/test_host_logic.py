@@ -1,0 +1,69 @@
+"""CPU-only checks of the library's host logic: exports, integer schedule, cache plan."""
+import os
+import re
+
+import pytest
+
+from oracle import skipdecode_oracle as O
+from paper_2307_02628_b200 import binding, synth
+
+
+def test_library_exports_every_declared_symbol(repo_root):
+    hdr = open(os.path.join(repo_root, "include", "skipdecode.h")).read()
+    declared = set(re.findall(r"\b(sd_[a-z_]+)\s*\(", hdr))
+    assert declared == set(binding.EXPORTS)
+    L = binding.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+SCHEDULES = [(4, 4, 2, 0, 32), (12, 12, 4, 0, 128), (24, 24, 8, 0, 256), (32, 32, 8, 0, 512), (32, 32, 4, 0, 1024),
+             (32, 22, 11, 1, 1024), (32, 14, 8, 1, 512), (32, 10, 6, 1, 100), (32, 8, 5, 1, 1024),
+             (24, 16, 8, 1, 512), (24, 10, 6, 1, 100), (24, 7, 5, 1, 37), (24, 6, 4, 1, 3),
+             (7, 7, 7, 0, 5), (9, 8, 2, 1, 1), (9, 8, 2, 1, 2), (40, 39, 3, 2, 2047)]
+
+
+@pytest.mark.parametrize("L,mx,mn,w,G", SCHEDULES)
+def test_schedule_is_bit_exact_with_the_oracle(L, mx, mn, w, G):
+    n, top = binding.schedule_compute(L, mx, mn, w, G)
+    n_ref, top_ref = O.schedule(mx, mn, w, G, L)
+    assert n == n_ref and top == top_ref
+
+
+@pytest.mark.parametrize("args", [(4, 5, 2, 0, 8), (8, 4, 5, 0, 8), (8, 4, 2, 2, 8), (8, 4, 2, 0, 0), (8, 4, 2, -1, 8)])
+def test_schedule_rejects_bad_arguments(args):
+    with pytest.raises(binding.SdError) as e:
+        binding.schedule_compute(*args)
+    assert e.value.code == binding.SD_ERR_ARG
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4", "c5"])
+def test_cache_plan_matches_the_active_sets(name):
+    wl = synth.CONFIGS[name]
+    cfg = binding.make_config(wl.shape, wl.batch, wl.prompt_len, wl.gen_len)
+    plan = binding.SdPlan(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len, 0)
+    cap = binding.layer_capacity(cfg, plan)
+    n, _ = O.schedule(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len, wl.shape.n_layers)
+    act = O.active_matrix(wl.shape.n_layers, wl.prompt_len, n, wl.warmup)
+    assert cap == [int(c) for c in act.sum(0)]          # positions at which each layer ever runs
+    full = binding.layer_capacity(cfg, binding.SdPlan(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len, 1))
+    assert full == [wl.prompt_len + wl.gen_len] * wl.shape.n_layers
+    e = 4 if wl.shape.dtype == "fp32" else 2
+    kv = 2 * sum(cap) * wl.batch * wl.shape.d_model * e
+    total = binding.arena_bytes(cfg, plan)
+    assert kv <= total <= kv + (2 << 30)                # caches dominate; activations and partials are bounded
+
+
+def test_config_validation():
+    shape = synth.TINY
+    plan = binding.SdPlan(4, 2, 0, 8, 0)
+    for bad in (dict(n_heads=3), dict(d_model=250), dict(max_prompt=100, max_gen=100), dict(dtype=2), dict(max_batch=0)):
+        cfg = binding.make_config(shape, 2, 8, 8)
+        for k, v in bad.items():
+            setattr(cfg, k, v)
+        with pytest.raises(binding.SdError):
+            binding.arena_bytes(cfg, plan)
+    cfg = binding.make_config(shape, 2, 8, 8)
+    with pytest.raises(binding.SdError):
+        binding.arena_bytes(cfg, binding.SdPlan(4, 2, 0, 9, 0))     # plan longer than max_gen
+    assert binding.lib().sd_strerror(binding.SD_ERR_POSITION).decode().startswith("position")
