@@ -141,6 +141,11 @@ int sd_prefill(sd_handle *h, const int32_t *d_tokens, int B, int P, float *d_log
  * Errors: SD_ERR_ARG, SD_ERR_STATE (no prefill), SD_ERR_POSITION, SD_ERR_CUDA. */
 int sd_decode_step(sd_handle *h, const int32_t *d_token_ids, int position, float *d_logits);
 
+/* Restarts generation at the end of the prompt: the next sd_decode_step must be at
+ * position P again.  The prompt's cache entries are kept; entries of generated
+ * positions are overwritten as the new steps reach them.  Errors: SD_ERR_STATE. */
+int sd_rewind(sd_handle *h);
+
 /* The same step with HOST buffers: copies h_token_ids [B] to the device, runs the
  * step, copies the logits [B, vocab] back and synchronises the stream.  Pinned
  * host memory makes the copies asynchronous to the host but is not required. */
@@ -158,6 +163,9 @@ int sd_status(sd_handle *h, int32_t *device_status);
 /* Decode steps run since sd_create and the number of layer executions they made
  * (their ratio is the mean active layers per generated token). */
 int sd_stats(sd_handle *h, int64_t *steps, int64_t *layer_steps);
+
+/* Kernels this handle has launched since sd_create (graph replays count their nodes). */
+int sd_launch_count(sd_handle *h, int64_t *launches);
 
 /* Tuning knobs; every value of every option computes the same function. */
 enum {

@@ -21,7 +21,7 @@ SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING = 1, 2, 3, 4
 KERNEL_CLASSES = ("embed", "layernorm", "gemm", "kv_append", "attention", "combine", "lm_head")
 
 EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_layer_capacity",
-           "sd_prefill", "sd_decode_step", "sd_decode_step_host", "sd_greedy", "sd_status", "sd_stats",
+           "sd_prefill", "sd_decode_step", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_status", "sd_stats",
            "sd_set_option", "sd_kernel_time", "sd_kernel_time_reset", "sd_strerror", "sd_destroy")
 
 
@@ -67,6 +67,8 @@ def lib() -> C.CDLL:
     L.sd_layer_capacity.argtypes = [C.POINTER(SdConfig), C.POINTER(SdPlan), i32p]
     L.sd_prefill.argtypes = [vp, vp, C.c_int, C.c_int, vp]
     L.sd_decode_step.argtypes = [vp, vp, C.c_int, vp]
+    L.sd_rewind.argtypes = [vp]
+    L.sd_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
     L.sd_decode_step_host.argtypes = [vp, vp, C.c_int, vp]
     L.sd_greedy.argtypes = [vp, vp, C.c_int, vp]
     L.sd_status.argtypes = [vp, i32p]
@@ -191,6 +193,14 @@ class Decoder:
         assert logits.dtype == torch.float32 and logits.is_contiguous() and ids.is_contiguous()
         _check(lib().sd_decode_step_host(self.h, ids.data_ptr(), position, logits.data_ptr()), "sd_decode_step_host")
         return logits
+
+    def rewind(self):
+        _check(lib().sd_rewind(self.h), "sd_rewind")
+
+    def launch_count(self) -> int:
+        v = C.c_int64(0)
+        _check(lib().sd_launch_count(self.h, C.byref(v)), "sd_launch_count")
+        return v.value
 
     # -- helpers ----------------------------------------------------------------------
     def greedy(self, logits: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:

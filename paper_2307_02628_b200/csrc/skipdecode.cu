@@ -51,11 +51,12 @@ struct sd_handle {
   int warmup = 0, gen_len = 0;
   bool have_schedule = false, have_prefill = false;
   int B = 0, P = 0, next_pos = 0;
-  int64_t steps = 0, layer_steps = 0;
+  int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
   int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0;
   // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
-  std::map<std::tuple<int, int, int, int, int, const void*, const void*>, cudaGraphExec_t> graphs;
+  struct Graph { cudaGraphExec_t exec; int64_t nodes; };
+  std::map<std::tuple<int, int, int, int, int, const void*, const void*>, Graph> graphs;
   // timing
   std::vector<Timed> timed;
   double k_ms[SD_K_COUNT] = {};
@@ -155,6 +156,7 @@ struct Launcher {
   sd_handle* h;
   bool timing;
   int err = 0;
+  int64_t count = 0;      // kernels enqueued through this launcher
   void begin(int cls) {
     if (!timing) return;
     Timed t; t.cls = cls;
@@ -163,6 +165,7 @@ struct Launcher {
     h->timed.push_back(t);
   }
   void end() {
+    ++count;
     if (cudaGetLastError() != cudaSuccess) err = SD_ERR_CUDA;
     if (timing) cudaEventRecord(h->timed.back().b, h->stream);
   }
@@ -284,7 +287,7 @@ int pick_chunk(const sd_handle* h, int rows, int T) {
 
 template <typename T>
 int enqueue_decode(sd_handle* h, const int32_t* d_ids, int pos, bool pos_from_device, float* d_logits, int n, int chunk,
-                   int n_chunks, bool timing) {
+                   int n_chunks, bool timing, int64_t* launched) {
   Launcher Lc{h, timing};
   const int L = h->cfg.n_layers, w = h->warmup, top = L - (n - w);
   sd::RowMap map{1, 0, pos, pos_from_device ? h->d_pos() : nullptr};
@@ -294,6 +297,7 @@ int enqueue_decode(sd_handle* h, const int32_t* d_ids, int pos, bool pos_from_de
     enqueue_layer<T>(Lc, l, h->B, map, chunk, n_chunks);
   }
   enqueue_head<T>(Lc, h->B, nullptr, d_logits);
+  *launched = Lc.count;
   return Lc.err;
 }
 
@@ -310,7 +314,9 @@ int run_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_lo
     for (int l = 0; l < L; ++l) enqueue_layer<T>(Lc, l, rows, map, chunk, 1);
     last_rows_kernel<<<(nb + 127) / 128, 128, 0, h->stream>>>(h->at<int>(h->A.row_index), nb, P);
     enqueue_head<T>(Lc, nb, h->at<int>(h->A.row_index), d_logits + (size_t)b0 * h->cfg.vocab);
+    Lc.count += 1;
   }
+  h->launches += Lc.count;
   return Lc.err;
 }
 
@@ -326,7 +332,7 @@ void collect_timing(sd_handle* h) {
 }
 
 void drop_graphs(sd_handle* h) {
-  for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+  for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second.exec);
   h->graphs.clear();
 }
 
@@ -341,10 +347,11 @@ int decode_step_impl(sd_handle* h, const int32_t* d_ids, int position, float* d_
   const int n_chunks = (T + chunk - 1) / chunk;
   const bool bf = h->cfg.dtype == SD_DTYPE_BF16;
   int err = 0;
+  int64_t launched = 0;
   const bool graphs = h->opt_graphs && !h->opt_timing && h->stream != nullptr;
   if (!graphs) {
-    err = bf ? enqueue_decode<bf16>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0)
-             : enqueue_decode<float>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0);
+    err = bf ? enqueue_decode<bf16>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0, &launched)
+             : enqueue_decode<float>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0, &launched);
   } else {
     auto key = std::make_tuple(h->B, n, h->warmup, chunk, n_chunks, (const void*)d_ids, (const void*)d_logits);
     auto it = h->graphs.find(key);
@@ -352,20 +359,22 @@ int decode_step_impl(sd_handle* h, const int32_t* d_ids, int position, float* d_
       if (h->graphs.size() >= 256) drop_graphs(h);
       cudaGraph_t graph = nullptr;
       if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
-      err = bf ? enqueue_decode<bf16>(h, d_ids, position, true, d_logits, n, chunk, n_chunks, false)
-               : enqueue_decode<float>(h, d_ids, position, true, d_logits, n, chunk, n_chunks, false);
+      err = bf ? enqueue_decode<bf16>(h, d_ids, position, true, d_logits, n, chunk, n_chunks, false, &launched)
+               : enqueue_decode<float>(h, d_ids, position, true, d_logits, n, chunk, n_chunks, false, &launched);
       const cudaError_t ce = cudaStreamEndCapture(h->stream, &graph);
       if (ce != cudaSuccess || err || !graph) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return SD_ERR_CUDA; }
       cudaGraphExec_t exec = nullptr;
       const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
       cudaGraphDestroy(graph);
       if (ie != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
-      it = h->graphs.emplace(key, exec).first;
+      it = h->graphs.emplace(key, sd_handle::Graph{exec, launched}).first;
     }
     set_int_kernel<<<1, 1, 0, h->stream>>>(h->d_pos(), position);
-    if (cudaGraphLaunch(it->second, h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+    if (cudaGraphLaunch(it->second.exec, h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+    launched = it->second.nodes + 1;
   }
   if (err) return err;
+  h->launches += launched;
   h->next_pos = position + 1;
   h->steps += 1;
   h->layer_steps += n;
@@ -471,6 +480,19 @@ int sd_decode_step(sd_handle* h, const int32_t* d_token_ids, int position, float
   return decode_step_impl(h, d_token_ids, position, d_logits);
 }
 
+int sd_rewind(sd_handle* h) {
+  if (!h) return SD_ERR_ARG;
+  if (!h->have_schedule || !h->have_prefill) return SD_ERR_STATE;
+  h->next_pos = h->P;
+  return SD_OK;
+}
+
+int sd_launch_count(sd_handle* h, int64_t* launches) {
+  if (!h || !launches) return SD_ERR_ARG;
+  *launches = h->launches;
+  return SD_OK;
+}
+
 int sd_decode_step_host(sd_handle* h, const int32_t* h_ids, int position, float* h_logits) {
   if (!h || !h_ids || !h_logits) return SD_ERR_ARG;
   if (!h->have_schedule || !h->have_prefill) return SD_ERR_STATE;
@@ -487,6 +509,7 @@ int sd_decode_step_host(sd_handle* h, const int32_t* h_ids, int position, float*
 int sd_greedy(sd_handle* h, const float* d_logits, int B, int32_t* d_next) {
   if (!h || !d_logits || !d_next || B < 1) return SD_ERR_ARG;
   sd::greedy_kernel<<<B, 1024, 0, h->stream>>>(d_logits, h->cfg.vocab, d_next);
+  h->launches += 1;
   return cudaGetLastError() == cudaSuccess ? SD_OK : SD_ERR_CUDA;
 }
 
