@@ -1,0 +1,357 @@
+"""Benchmark: skip-decode tokens/s of an OPT-shaped decoder on B200, with its roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c4] [--impl ours|reference]
+
+One "step" is one pass of the whole decode path over one batch: gen_len calls of
+sd_decode_step (every position of the budget schedule, the greedy pick between
+them) starting from the prompt's cache.  The prompt is processed once, untimed.
+`value` = batch * gen_len * N / seconds per step, timed on the device with the
+inputs resident in HBM; `e2e` is the same loop through sd_decode_step_host with
+pinned HOST buffers (token ids in, logits out, every step).
+
+With N > 1 (torchrun) every rank runs an independent replica of the workload on
+its own GPU: the path has no exchange step, so no collective is in the timed
+region; the barrier and the max over ranks use NCCL.
+
+--impl reference times the CPU oracle as it stands on the host cores, on a bounded
+sample of the same workload (a few batch rows, a few decode steps per "step").
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2307_02628_b200 import synth  # noqa: E402
+
+METRIC = "decode tokens/s at OPT-6.7B shape bs64 (% roofline); speedup vs full-layer"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------- byte model
+
+def layer_weight_bytes(shape: synth.ModelShape) -> int:
+    d, f = shape.d_model, shape.d_ffn
+    e = 4 if shape.dtype == "fp32" else 2
+    return (4 * d * d + 2 * d * f + 9 * d + f) * e
+
+
+def step_bytes(wl: synth.Workload, n_active) -> float:
+    """Algorithmic bytes of one pass: per decode step n (W_layer + K,V read) + LM head + logits."""
+    s = wl.shape
+    e = 4 if s.dtype == "fp32" else 2
+    total = 0.0
+    for g, n in enumerate(n_active):
+        T = wl.prompt_len + g + 1
+        total += n * (layer_weight_bytes(s) + 2.0 * T * s.d_model * wl.batch * e)
+        total += s.vocab * s.d_model * e + wl.batch * s.vocab * 4
+    return total
+
+
+# --------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.rows, self.proc = [], None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.cmd = ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "200"]
+        except Exception:
+            self.cmd = None
+
+    def start(self):
+        if not self.cmd:
+            return
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for nm, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            except Exception:
+                continue
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+
+def oracle_sample(wl: synth.Workload, weights, rows: int, steps_per_call: int, calls: int, warm_calls: int):
+    """Times the oracle's cached decode steps on `rows` batch rows: returns (tokens/s, seconds per call)."""
+    from oracle import skipdecode_oracle as O
+    prompts = synth.make_prompts(wl)[:rows]
+    dec = O.CachedDecoder(weights, wl.shape.n_heads, torch.float32)
+    dec.set_schedule(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len)
+    logits = dec.prefill(prompts)
+    pos = wl.prompt_len
+    times = []
+    for c in range(warm_calls + calls):
+        t0 = time.perf_counter()
+        for _ in range(steps_per_call):
+            if pos - wl.prompt_len >= wl.gen_len:
+                break
+            ids = O.greedy(logits)
+            logits = dec.decode_step(ids, pos)
+            pos += 1
+        dt = time.perf_counter() - t0
+        if c >= warm_calls:
+            times.append(dt)
+    sec = sum(times) / max(1, len(times))
+    return rows * steps_per_call / sec, sec
+
+
+def reference_arm(args, wl, rank):
+    if rank != 0:
+        return
+    cores = torch.get_num_threads()
+    weights = synth.make_weights(wl.shape, seed=0, threads=cores)
+    rows, spc = args.ref_rows, args.ref_steps
+    tps, sec = oracle_sample(wl, weights, rows, spc, args.steps, args.warmup)
+    sample = f"{rows} batch row(s), {spc} decode step(s) per timed step from position {wl.prompt_len}, fp32, after an untimed prompt pass"
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": bench_config(wl, args),
+            "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def bench_config(wl, args):
+    s = wl.shape
+    return {"workload": f"{args.config}: {s.name} L{s.n_layers} d{s.d_model} H{s.n_heads} f{s.d_ffn} V{s.vocab} {s.dtype}, "
+                        f"batch {wl.batch}, prompt {wl.prompt_len}, gen {wl.gen_len}, linear budget {wl.max_layers}->{wl.min_layers} top layers, warm-up {wl.warmup}",
+            "global_batch": wl.batch * args.gpus, "l2": "inputs larger than L2 (KV cache and weights are GBs)",
+            "tokens": "greedy on device (value); forced ids from host (e2e)"}
+
+
+# --------------------------------------------------------------------------- GPU arm
+
+def gpu_arm(args, wl, rank, world):
+    from paper_2307_02628_b200 import binding
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    device = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist_.init_process_group("nccl", device_id=device)
+        dist = dist_
+    s, B, P, G = wl.shape, wl.batch, wl.prompt_len, wl.gen_len
+    t0 = time.perf_counter()
+    weights = synth.make_weights(s, seed=0, threads=torch.get_num_threads())
+    t_weights = time.perf_counter() - t0
+
+    free, _total = torch.cuda.mem_get_info(device)
+    wbytes = sum(t.numel() * t.element_size() for t in [weights["tok_emb"], weights["pos_emb"]] +
+                 [t for lw in weights["layers"] for t in lw.values()])
+    cfg = binding.make_config(s, B, P, G)
+    need_full = binding.arena_bytes(cfg, binding.SdPlan(wl.max_layers, wl.min_layers, wl.warmup, G, 1))
+    full_ok = (not args.no_full_layer) and need_full + wbytes + (4 << 30) < free
+    dec = binding.Decoder(s, weights, B, P, G, plan=(wl.max_layers, wl.min_layers, wl.warmup, G),
+                          full_capacity=full_ok, device=str(device))
+    stream = dec.stream
+    prompts = synth.make_prompts(wl).to(device)
+    forced = synth.make_forced_tokens(wl)
+    logits0 = torch.empty(B, s.vocab, dtype=torch.float32, device=device)
+    logits = torch.empty(B, s.vocab, dtype=torch.float32, device=device)
+    ids = torch.empty(B, dtype=torch.int32, device=device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    def one_pass():
+        dec.rewind()
+        dec.greedy(logits0, ids)
+        for g in range(G):
+            dec.decode_step(ids, P + g, logits)
+            dec.greedy(logits, ids)
+
+    def timed(fn, reps):
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        barrier()
+        ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / reps
+
+    with torch.cuda.stream(stream):
+        n_active, _ = dec.schedule(wl.max_layers, wl.min_layers, wl.warmup, G)
+        tp0 = time.perf_counter()
+        dec.prefill(prompts, logits0)
+        stream.synchronize()
+        t_prefill = time.perf_counter() - tp0
+
+        for _ in range(args.warmup):
+            one_pass()
+        clocks = ClockSampler(device)
+        clocks.start()
+        l0 = dec.launch_count()
+        ms_step = timed(one_pass, args.steps)
+        launches = dec.launch_count() - l0
+        clock_info = clocks.stop()
+        assert dec.status() == 0, "device status word set"
+
+        # end to end: host ids in, logits out, every step, through sd_decode_step_host
+        h_ids = forced.t().contiguous().pin_memory()            # [G, B]
+        h_logits = torch.empty(B, s.vocab, dtype=torch.float32).pin_memory()
+
+        def e2e_pass():
+            dec.rewind()
+            for g in range(G):
+                dec.decode_step_host(h_ids[g], P + g, h_logits)
+
+        e2e_pass()
+        barrier()
+        te = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_pass()
+        barrier()
+        e2e_s = (time.perf_counter() - te) / args.e2e_steps
+        if dist is not None:
+            t = torch.tensor([e2e_s], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+
+        # dominant kernel (decode attention): device time per launch on sampled steps
+        dec.rewind()
+        dec.kernel_times_reset()
+        dec.greedy(logits0, ids)
+        attn_bytes = 0.0
+        e = 4 if s.dtype == "fp32" else 2
+        for g in range(G):
+            sampled = (g % args.profile_every == 0)
+            dec.set_option(binding.SD_OPT_TIMING, 1 if sampled else 0)
+            dec.decode_step(ids, P + g, logits)
+            dec.greedy(logits, ids)
+            if sampled:
+                attn_bytes += n_active[g] * 2.0 * (P + g + 1) * s.d_model * B * e
+        dec.set_option(binding.SD_OPT_TIMING, 0)
+        kt = dec.kernel_times()
+        attn_ms, attn_n = kt["attention"]
+
+        full = None
+        if full_ok:
+            dec.schedule(s.n_layers, s.n_layers, 0, G)
+            one_pass()
+            ms_full = timed(one_pass, max(1, min(2, args.steps)))
+            full = {"ms_per_step": ms_full, "tokens_per_s": world * B * G / (ms_full / 1e3),
+                    "speedup_skip_over_full": ms_full / ms_step,
+                    "byte_model_bound": step_bytes(wl, [s.n_layers] * G) / step_bytes(wl, n_active)}
+
+    peak, peak_kind = measured_peaks()
+    value = world * B * G / (ms_step / 1e3)
+    total_bytes = step_bytes(wl, n_active)
+    achieved = attn_bytes / (attn_ms / 1e3) / 1e9 if attn_ms > 0 else None
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic", "config": bench_config(wl, args),
+        "clocks": clock_info, "gpu_launches": int(launches),
+        "e2e": {"value": world * B * G / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": G * B * 4,
+                "d2h_bytes_per_step": G * B * s.vocab * 4},
+        "roofline": {"kernel": "attn_partial_kernel (split-KV decode attention)", "bound": "hbm", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
+                     "traffic": None, "launches_timed": int(attn_n),
+                     "algorithmic_bytes_per_launch": attn_bytes / attn_n if attn_n else None},
+        "step_roofline": {"algorithmic_bytes_per_step": total_bytes, "achieved_gbs": total_bytes / (ms_step / 1e3) / 1e9,
+                          "frac_of_measured_hbm": total_bytes / (ms_step / 1e3) / 1e9 / peak,
+                          "frac_of_8tbs": total_bytes / (ms_step / 1e3) / 1e9 / 8000.0},
+        "kernel_time_share": {k: v[0] for k, v in kt.items()},
+        "full_layer": full, "prefill_s": t_prefill, "weights_s": t_weights,
+        "mean_active_layers": sum(n_active) / len(n_active),
+    }
+    dec.close()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cores = torch.get_num_threads()
+        tps, sec = oracle_sample(wl, weights, args.ref_rows, args.ref_steps, 2, 1)
+        line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                                "sample": f"{args.ref_rows} batch row(s), 2 timed calls of {args.ref_steps} decode step(s) from position {P}, fp32, after an untimed prompt pass"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c4", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--profile-every", type=int, default=8)
+    ap.add_argument("--no-full-layer", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-rows", type=int, default=1)
+    ap.add_argument("--ref-steps", type=int, default=1)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    wl = synth.CONFIGS[args.config]
+    if args.impl == "reference":
+        reference_arm(args, wl, rank)
+        return
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torchrun for N > 1")
+    gpu_arm(args, wl, rank, world)
+
+
+if __name__ == "__main__":
+    main()

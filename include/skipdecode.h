@@ -113,7 +113,9 @@ int sd_create(const sd_config *cfg, const sd_weights *weights, const sd_plan *pl
  * n_active, top_begin: host, gen_len int32 each, either may be NULL.
  * Requires 0 <= warmup < min_layers <= max_layers <= n_layers, 1 <= gen_len <= max_gen.
  * Errors: SD_ERR_ARG; SD_ERR_CAPACITY if a layer would need more cache positions
- * than the plan given to sd_create reserved.  Resets the sequence state. */
+ * than the plan given to sd_create reserved.  Generation restarts at the end of the
+ * prompt: a prompt already processed by sd_prefill stays valid (its cache entries do
+ * not depend on the schedule) unless P + gen_len now exceeds max_pos. */
 int sd_schedule(sd_handle *h, int max_layers, int min_layers, int warmup, int gen_len,
                 int32_t *n_active, int32_t *top_begin);
 

@@ -443,7 +443,10 @@ int sd_schedule(sd_handle* h, int mx, int mn, int w, int G, int32_t* n_active, i
     if (top_begin) top_begin[g] = h->top_begin[g];
   }
   h->warmup = w; h->gen_len = G;
-  h->have_schedule = true; h->have_prefill = false;
+  h->have_schedule = true;
+  // the prompt's cache does not depend on the schedule: keep it when the new length still fits
+  if (h->have_prefill && (int64_t)h->P + G > h->cfg.max_pos) h->have_prefill = false;
+  h->next_pos = h->P;
   return SD_OK;
 }
 
