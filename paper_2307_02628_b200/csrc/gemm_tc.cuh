@@ -1,19 +1,339 @@
-// Tensor-core GEMM for bf16 operands (placeholder: not taken yet, every call falls
-// through to the CUDA-core kernel).
+// Tensor-core GEMM for bf16 operands on sm_100a: out[m, n] (+)= sum_k X[m, k] W[n, k] + bias[n].
+//
+// The weight's output dimension sits on the MMA M axis (D^T = W X^T): a CTA owns 128 rows
+// of W, so tiles are full even when the token count M is 16..256, which becomes the MMA N.
+// Operands reach shared memory by TMA (128-byte swizzle, K-major, no multicast), the
+// accumulator lives in tensor memory, and one thread issues tcgen05.mma.  Warp roles:
+// warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue (each
+// reads its own quarter of the 128 TMEM lanes).  K can be split over blockIdx.z for the
+// residual epilogue, whose partial sums are added to the fp32 residual stream atomically.
+//
+// Every mbarrier wait is bounded: on expiry the CTA raises an abort flag, records
+// STATUS_WAIT_EXPIRED in the status word, drains the copies it issued and frees its TMEM.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <map>
+#include <tuple>
+
+#include "kernels.cuh"
+
 namespace sd {
 
-struct TcContext { int ready = 0; };
-inline void tc_init(TcContext&) {}
-inline void tc_destroy(TcContext&) {}
+namespace tc {
 
-// Returns true when the product was enqueued on the tensor-core path.
+constexpr int BM = 128;              // W rows (output features) per CTA = MMA M
+constexpr int BK = 64;               // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr long long kWaitLimit = 4000000000LL;   // clock cycles (~2 s) before a wait gives up
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this or another wait expired).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimit) {
+      *abort_flag = 1;
+      atomicOr(status, STATUS_WAIT_EXPIRED);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// K-major operand tile in shared memory, rows of 128 bytes, 128-byte swizzle, groups of 8
+// rows 1024 bytes apart.  Fields: start address >> 4 [0,14), leading byte offset >> 4
+// [16,30) (unused for swizzled K-major, set to 1), stride byte offset >> 4 [32,46) = 64,
+// descriptor version 1 [46,48), layout type 2 = SWIZZLE_128B [61,64).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// kind::f16 instruction descriptor: D = fp32 [4,6), A = B = bf16 [7,10) [10,13), both K-major,
+// N >> 3 at [17,23), M >> 4 at [24,29).
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+
+__host__ __device__ constexpr int stages_for(int nb) { return nb >= 256 ? 4 : nb >= 128 ? 6 : 8; }
+__host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + nb * BK * 2; }
+__host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/; }
+
+template <int NB, int EPI>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+               const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
+               int kb_per_split, int* __restrict__ status) {
+  constexpr int STAGES = stages_for(NB);
+  constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2;
+  constexpr int TMEM_COLS = NB < 32 ? 32 : NB;
+  constexpr int CW = NB < 32 ? 16 : 32;          // accumulator columns read per tcgen05.ld
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                 // swizzled tiles need 1024-byte alignment
+  uint8_t* tiles_ptr = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * (A_BYTES + B_BYTES));
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * STAGES, accum_bar = full0 + 16 * STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * BM, m0 = blockIdx.y * NB;
+  const int kb_total = (K + BK - 1) / BK;
+  const int kb0 = blockIdx.z * kb_per_split, kb1 = min(kb0 + kb_per_split, kb_total);
+  const int nkb = kb1 - kb0;                                     // >= 1 by construction of the grid
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(accum_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+      int issued = 0;
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % STAGES, round = i / STAGES;
+        if (round > 0 && !mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
+        const uint32_t fb = full0 + 8 * s;
+        mbar_expect_tx(fb, A_BYTES + B_BYTES);
+        const uint32_t a_dst = tiles + s * (A_BYTES + B_BYTES);
+        tma_load_2d(a_dst, &map_w, (kb0 + i) * BK, n0, fb);
+        tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);
+        issued = i + 1;
+      }
+      if (*abort_flag) {
+        // drain: wait (bounded) until every copy issued has landed before the CTA exits
+        const int first = issued > STAGES ? issued - STAGES : 0;
+        for (int i = first; i < issued; ++i) {
+          const long long t0 = clock64();
+          while (!mbar_try(full0 + 8 * (i % STAGES), (i / STAGES) & 1) && clock64() - t0 < kWaitLimit) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(NB);
+      bool ok = true;
+      for (int i = 0; i < nkb && ok; ++i) {
+        const int s = i % STAGES, round = i / STAGES;
+        ok = mbar_wait(full0 + 8 * s, round & 1, abort_flag, status);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = tiles + s * (A_BYTES + B_BYTES);
+        const uint64_t a_desc = smem_desc(a_addr), b_desc = smem_desc(a_addr + A_BYTES);
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k)     // 32 bytes further along K inside the swizzle row
+          umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+        umma_commit(empty0 + 8 * s);              // the stage is free once these MMAs have read it
+      }
+      if (ok) umma_commit(accum_bar);             // accumulator complete
+    }
+  } else {
+    const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, +32) belong to this warp
+    const int n = n0 + quarter * 32 + lane;
+    if (mbar_wait(accum_bar, 0, abort_flag, status)) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const float b = (bias != nullptr && n < N && (EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
+#pragma unroll 1
+      for (int c = 0; c < NB; c += CW) {
+        uint32_t r[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
+        if (CW == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (n < N) {
+#pragma unroll
+          for (int j = 0; j < CW; ++j) {
+            const int m = m0 + c + j;
+            if (m < M) {
+              const float v = __uint_as_float(r[j]) + b;
+              const size_t idx = (size_t)m * ldo + n;
+              if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
+              else if (EPI == EPI_RELU_T) reinterpret_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(fmaxf(v, 0.f));
+              else atomicAdd(reinterpret_cast<float*>(out) + idx, v);
+            }
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace tc
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcContext {
+  EncodeTiledFn encode = nullptr;
+  int ready = 0;
+  int sm_count = 148;
+  // (pointer, rows, cols, box rows) -> tensor map of a row-major bf16 matrix, 64-column boxes, 128-byte swizzle
+  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
+};
+
+template <int NB, int EPI>
+inline bool tc_prepare() {
+  return cudaFuncSetAttribute(tc::gemm_tc_kernel<NB, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(NB)) == cudaSuccess;
+}
+template <int NB>
+inline bool tc_prepare_nb() {
+  return tc_prepare<NB, EPI_STORE_F32>() && tc_prepare<NB, EPI_RELU_T>() && tc_prepare<NB, EPI_RESIDUAL_F32>();
+}
+
+inline void tc_init(TcContext& c) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+      q != cudaDriverEntryPointSuccess) {
+    cudaGetLastError();
+    return;
+  }
+  c.encode = reinterpret_cast<EncodeTiledFn>(fn);
+  int dev = 0, major = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return; }
+  cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (major != 10) return;                       // tcgen05 exists on sm_100 only
+  if (sms > 0) c.sm_count = sms;
+  if (!(tc_prepare_nb<16>() && tc_prepare_nb<32>() && tc_prepare_nb<64>() && tc_prepare_nb<128>() && tc_prepare_nb<256>())) {
+    cudaGetLastError();
+    return;
+  }
+  c.ready = 1;
+}
+inline void tc_destroy(TcContext& c) { c.maps.clear(); c.ready = 0; }
+
+inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int cols, int box_rows) {
+  auto key = std::make_tuple(ptr, rows, cols, box_rows);
+  auto it = c.maps.find(key);
+  if (it != c.maps.end()) return &it->second;
+  CUtensorMap m;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  if (c.encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return nullptr;
+  if (c.maps.size() > 4096) c.maps.clear();
+  return &c.maps.emplace(key, m).first->second;
+}
+
+template <int NB>
+inline bool tc_launch(cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
+                      int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status) {
+  dim3 grid((N + tc::BM - 1) / tc::BM, (M + NB - 1) / NB, splits);
+  const int smem = tc::smem_bytes(NB);
+  if (epi == EPI_STORE_F32)
+    tc::gemm_tc_kernel<NB, EPI_STORE_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status);
+  else if (epi == EPI_RELU_T)
+    tc::gemm_tc_kernel<NB, EPI_RELU_T><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status);
+  else
+    tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status);
+  return true;
+}
+
+// Returns true when the product was enqueued on the tensor-core path; false leaves it to the caller.
+inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const __nv_bfloat16* W, const __nv_bfloat16* bias,
+                    int M, int N, int K, void* out, int ldo, int epi, int* status) {
+  if (!c.ready || K % 8 || M < 1 || N < 1) return false;
+  if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
+  const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+  const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
+  const CUtensorMap* mx = tc_map(c, X, M, K, nb);
+  if (!mw || !mx) return false;
+  const int kb_total = (K + tc::BK - 1) / tc::BK;
+  int splits = 1;
+  if (epi == EPI_RESIDUAL_F32) {                 // partial sums may be added in any order
+    const int tiles = ((N + tc::BM - 1) / tc::BM) * ((M + nb - 1) / nb);
+    splits = std::max(1, std::min(kb_total / 4, (c.sm_count + tiles - 1) / tiles));
+  }
+  int kb_per_split = (kb_total + splits - 1) / splits;
+  splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split
+  switch (nb) {
+    case 16: return tc_launch<16>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
+    case 32: return tc_launch<32>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
+    case 64: return tc_launch<64>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
+    case 128: return tc_launch<128>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
+    default: return tc_launch<256>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
+  }
+}
 template <typename T>
 inline bool tc_gemm(TcContext&, cudaStream_t, const T*, const T*, const T*, int, int, int, void*, int, int, int*) {
-  return false;
+  return false;                                  // fp32 storage runs on the CUDA-core kernel
 }
 
 }  // namespace sd

@@ -196,3 +196,24 @@ def test_errors_are_reported_not_fatal():
         dec.decode_step(bad, 33)                                     # flagged on the device, clamped, no fault
         assert dec.status() == 1
     dec.close()
+
+
+@pytest.mark.parametrize("B,P", [(3, 37), (20, 9), (70, 5), (130, 3)])
+def test_tensor_core_and_cuda_core_gemm_paths_agree(B, P):
+    """bf16 products on the tcgen05 path against the same products on CUDA cores: every
+    token-tile width (16..256), ragged feature tiles (vocab 777, d_ffn 384) and split K."""
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("toy-gemm", 2, 256, 4, 384, 777, 64, "bf16")
+    wl = synth.Workload(shape, B, P, 6, 2, 1, 0)
+    w = synth.make_weights(shape, seed=8, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced)
+    outs = []
+    for mode in (1, 0):
+        dec = harness.make_decoder(wl, w)
+        dec.set_option(binding.SD_OPT_GEMM, mode)
+        outs.append(harness.gpu_run_forced(dec, wl, prompts, forced))
+        dec.close()
+        _check(outs[-1], ref, "bf16", f"gemm mode {mode} B{B} P{P}")
+    # same bf16 operands, fp32 accumulation in a different order
+    assert float((outs[0] - outs[1]).abs().max()) < 2e-3
