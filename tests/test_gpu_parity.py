@@ -216,4 +216,5 @@ def test_tensor_core_and_cuda_core_gemm_paths_agree(B, P):
         dec.close()
         _check(outs[-1], ref, "bf16", f"gemm mode {mode} B{B} P{P}")
     # same bf16 operands, fp32 accumulation in a different order
-    assert float((outs[0] - outs[1]).abs().max()) < 2e-3
+    # a different summation order flips some bf16 roundings of the activations: ulp-scale differences
+    assert float((outs[0] - outs[1]).abs().max()) < 1e-2
