@@ -155,6 +155,8 @@ __global__ void last_rows_kernel(int* idx, int n, int P) {
 struct Launcher {
   sd_handle* h;
   bool timing;
+  float* part_acc;        // split-KV partial accumulators and (max, sum) pairs of this launch sequence
+  float* part_ml;
   int err = 0;
   int64_t count = 0;      // kernels enqueued through this launcher
   void begin(int cls) {
@@ -199,12 +201,11 @@ void launch_attention_hd(Launcher& Lc, const T* Kc, const T* Vc, int cap, int ro
   Lc.begin(SD_K_ATTENTION);
   dim3 grid(rows * H, n_chunks);
   sd::attn_partial_kernel<T, HD, 4><<<grid, 128, 0, h->stream>>>(
-      h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks,
-      h->at<float>(h->A.part_acc), h->at<float>(h->A.part_ml));
+      h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml);
   Lc.end();
   Lc.begin(SD_K_COMBINE);
   sd::attn_combine_kernel<T, HD><<<rows * H, HD < 64 ? 32 : 64, 0, h->stream>>>(
-      h->at<float>(h->A.part_acc), h->at<float>(h->A.part_ml), h->at<T>(h->A.o), H, cap, map, chunk, n_chunks);
+      Lc.part_acc, Lc.part_ml, h->at<T>(h->A.o), H, cap, map, chunk, n_chunks);
   Lc.end();
 }
 
@@ -287,8 +288,8 @@ int pick_chunk(const sd_handle* h, int rows, int T) {
 
 template <typename T>
 int enqueue_decode(sd_handle* h, const int32_t* d_ids, int pos, bool pos_from_device, float* d_logits, int n, int chunk,
-                   int n_chunks, bool timing, int64_t* launched) {
-  Launcher Lc{h, timing};
+                   int n_chunks, bool timing, int64_t* launched, float* part_acc = nullptr, float* part_ml = nullptr) {
+  Launcher Lc{h, timing, part_acc ? part_acc : h->at<float>(h->A.part_acc), part_ml ? part_ml : h->at<float>(h->A.part_ml)};
   const int L = h->cfg.n_layers, w = h->warmup, top = L - (n - w);
   sd::RowMap map{1, 0, pos, pos_from_device ? h->d_pos() : nullptr};
   enqueue_embed<T>(Lc, d_ids, h->B, map);
@@ -303,7 +304,7 @@ int enqueue_decode(sd_handle* h, const int32_t* d_ids, int pos, bool pos_from_de
 
 template <typename T>
 int run_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_logits) {
-  Launcher Lc{h, h->opt_timing != 0};
+  Launcher Lc{h, h->opt_timing != 0, h->at<float>(h->A.part_acc), h->at<float>(h->A.part_ml)};
   const int L = h->cfg.n_layers;
   const int per = std::max(1, kPrefillTokens / P);
   for (int b0 = 0; b0 < B; b0 += per) {
