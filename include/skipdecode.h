@@ -143,6 +143,35 @@ int sd_prefill(sd_handle *h, const int32_t *d_tokens, int B, int P, float *d_log
  * Errors: SD_ERR_ARG, SD_ERR_STATE (no prefill), SD_ERR_POSITION, SD_ERR_CUDA. */
 int sd_decode_step(sd_handle *h, const int32_t *d_token_ids, int position, float *d_logits);
 
+/* sd_decode_step with the split-KV attention's partial results kept in an array that is
+ * part of the library image instead of the caller's arena.  The paper has no counterpart
+ * to this call; it exists for callers that must not, or cannot, allocate device memory
+ * while they run: a plug-in loaded into a process whose device memory is owned and
+ * fully committed by its host application, a serving or real-time loop that forbids
+ * allocation after start-up, a process whose allocator is not reentrant from the thread
+ * that drives decoding.  Such a caller
+ * still passes the inputs and outputs (and the handle built at start-up); this call itself
+ * calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - The array holds SD_STATIC_SCRATCH_BYTES per GPU, resident on every GPU that loads
+ *     the library until the process exits.  A step needs
+ *       B * n_heads * ceil((position + 1) / chunk) * (head_dim + 2) * 4 bytes
+ *     (chunk = keys per attention split, see SD_OPT_ATTN_CHUNK); a step that needs more
+ *     fails with SD_ERR_CAPACITY and enqueues nothing.
+ *   - The first call on each device looks up the array's device address (one host-side
+ *     runtime query, with that device current).  Make that first call outside any stream
+ *     capture; later calls do no set-up.
+ *   - The CUDA device current on the calling thread must be the one that holds the handle's
+ *     arena; otherwise SD_ERR_ARG.
+ *   - All handles and all calls on one GPU share the array and it keeps the previous
+ *     call's contents.  Nothing in it needs clearing: each slot is written before it is
+ *     read within the same step.  Two such steps that overlap in time on one GPU (two
+ *     handles on two streams) overwrite each other's partial results: serialise them.
+ *   - Always plain kernel launches (SD_OPT_GRAPHS is ignored); SD_OPT_TIMING is not recorded.
+ * Arguments, ordering rules, results and errors are otherwise those of sd_decode_step,
+ * and the two calls may be mixed freely within one sequence. */
+#define SD_STATIC_SCRATCH_BYTES (16u << 20)
+int sd_decode_step_static(sd_handle *h, const int32_t *d_token_ids, int position, float *d_logits);
+
 /* Restarts generation at the end of the prompt: the next sd_decode_step must be at
  * position P again.  The prompt's cache entries are kept; entries of generated
  * positions are overwritten as the new steps reach them.  Errors: SD_ERR_STATE. */

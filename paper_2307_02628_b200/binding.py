@@ -21,7 +21,7 @@ SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING = 1, 2, 3, 4
 KERNEL_CLASSES = ("embed", "layernorm", "gemm", "kv_append", "attention", "combine", "lm_head")
 
 EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_layer_capacity",
-           "sd_prefill", "sd_decode_step", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_status", "sd_stats",
+           "sd_prefill", "sd_decode_step", "sd_decode_step_static", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_status", "sd_stats",
            "sd_set_option", "sd_kernel_time", "sd_kernel_time_reset", "sd_strerror", "sd_destroy")
 
 
@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
     L.sd_layer_capacity.argtypes = [C.POINTER(SdConfig), C.POINTER(SdPlan), i32p]
     L.sd_prefill.argtypes = [vp, vp, C.c_int, C.c_int, vp]
     L.sd_decode_step.argtypes = [vp, vp, C.c_int, vp]
+    L.sd_decode_step_static.argtypes = [vp, vp, C.c_int, vp]
     L.sd_rewind.argtypes = [vp]
     L.sd_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
     L.sd_decode_step_host.argtypes = [vp, vp, C.c_int, vp]
@@ -184,6 +185,18 @@ class Decoder:
             logits = torch.empty(ids.shape[0], self.shape.vocab, dtype=torch.float32, device=self.device)
         self._order()
         _check(lib().sd_decode_step(self.h, ids.data_ptr(), position, logits.data_ptr()), "sd_decode_step")
+        self._keep_io = (ids, logits)
+        return logits
+
+    def decode_step_static(self, ids: torch.Tensor, position: int, logits: torch.Tensor | None = None) -> torch.Tensor:
+        """sd_decode_step_static: the same step with the attention partials in the library's
+        own static device array, for callers that may not allocate (the tensors passed here
+        must already exist: this wrapper allocates `logits` only when it is not given)."""
+        ids = self._dev_i32(ids)
+        if logits is None:
+            logits = torch.empty(ids.shape[0], self.shape.vocab, dtype=torch.float32, device=self.device)
+        self._order()
+        _check(lib().sd_decode_step_static(self.h, ids.data_ptr(), position, logits.data_ptr()), "sd_decode_step_static")
         self._keep_io = (ids, logits)
         return logits
 

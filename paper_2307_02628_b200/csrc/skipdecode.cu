@@ -382,6 +382,26 @@ int decode_step_impl(sd_handle* h, const int32_t* d_ids, int position, float* d_
   return SD_OK;
 }
 
+// ---- static scratch for sd_decode_step_static -------------------------------------------
+// Lives in the library image: every GPU that loads the library holds these bytes until the
+// process exits.  In host code the symbol below is only a stand-in; the device address comes
+// from cudaGetSymbolAddress, looked up once per device with that device current.
+constexpr size_t kStaticScratchBytes = SD_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};
+
+int static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return SD_ERR_ARG;
+  if (!g_static_scratch_addr[device]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return SD_ERR_CUDA; }
+    g_static_scratch_addr[device] = p;
+  }
+  *out = g_static_scratch_addr[device];
+  return SD_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -494,6 +514,41 @@ int sd_rewind(sd_handle* h) {
 int sd_launch_count(sd_handle* h, int64_t* launches) {
   if (!h || !launches) return SD_ERR_ARG;
   *launches = h->launches;
+  return SD_OK;
+}
+
+int sd_decode_step_static(sd_handle* h, const int32_t* d_ids, int position, float* d_logits) {
+  if (!h || !d_ids || !d_logits) return SD_ERR_ARG;
+  if (!h->have_schedule || !h->have_prefill) return SD_ERR_STATE;
+  const int g = position - h->P;
+  if (position != h->next_pos || g < 0 || g >= h->gen_len || position >= h->cfg.max_pos) return SD_ERR_POSITION;
+  int device = -1;
+  cudaPointerAttributes attr;
+  if (cudaGetDevice(&device) != cudaSuccess || cudaPointerGetAttributes(&attr, h->arena) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  if (attr.device != device) return SD_ERR_ARG;       // the static array of another GPU would be handed to this handle's kernels
+  const int n = h->n_active[g];
+  const int T = position + 1;
+  const int chunk = pick_chunk(h, h->B, T);
+  const int n_chunks = (T + chunk - 1) / chunk;
+  const size_t slots = (size_t)h->B * h->cfg.n_heads * n_chunks;
+  const size_t acc_bytes = align_up(slots * h->hd * sizeof(float)), ml_bytes = slots * 2 * sizeof(float);
+  if (acc_bytes + ml_bytes > kStaticScratchBytes) return SD_ERR_CAPACITY;   // split-KV partials beyond the static array
+  void* base = nullptr;
+  const int rc = static_scratch_address(device, &base);
+  if (rc != SD_OK) return rc;
+  float* part_acc = static_cast<float*>(base);
+  float* part_ml = reinterpret_cast<float*>(static_cast<char*>(base) + acc_bytes);
+  int64_t launched = 0;
+  // every partial slot the combine kernel reads is written by the attention kernel of the same
+  // layer first, so nothing in the array has to start at zero
+  const int err = h->cfg.dtype == SD_DTYPE_BF16
+      ? enqueue_decode<bf16>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, false, &launched, part_acc, part_ml)
+      : enqueue_decode<float>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, false, &launched, part_acc, part_ml);
+  if (err) return err;
+  h->launches += launched;
+  h->next_pos = position + 1;
+  h->steps += 1;
+  h->layer_steps += n;
   return SD_OK;
 }
 
