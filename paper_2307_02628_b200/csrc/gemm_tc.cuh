@@ -1,4 +1,6 @@
 // Tensor-core GEMM for bf16 operands on sm_100a: out[m, n] (+)= sum_k X[m, k] W[n, k] + bias[n].
+// X is an Operand row (kernels.cuh): X = Xhi + Xlo, two bf16 matrices side by side in one
+// [M, 2K] buffer; both are multiplied with the same W tile into the same accumulator.
 //
 // The weight's output dimension sits on the MMA M axis (D^T = W X^T): a CTA owns 128 rows
 // of W, so tiles are full even when the token count M is 16..256, which becomes the MMA N.
@@ -107,8 +109,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr) : "memory");
 }
 
-__host__ __device__ constexpr int stages_for(int nb) { return nb >= 256 ? 4 : nb >= 128 ? 6 : 8; }
-__host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + nb * BK * 2; }
+__host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
+__host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/; }
 
 template <int NB, int EPI>
@@ -117,7 +119,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                int kb_per_split, int* __restrict__ status) {
   constexpr int STAGES = stages_for(NB);
-  constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2;
+  constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
   constexpr int TMEM_COLS = NB < 32 ? 32 : NB;
   constexpr int CW = NB < 32 ? 16 : 32;          // accumulator columns read per tcgen05.ld
 
@@ -125,7 +127,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                 // swizzled tiles need 1024-byte alignment
   uint8_t* tiles_ptr = smem_raw + (tiles - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * (A_BYTES + B_BYTES));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * STAGES, accum_bar = full0 + 16 * STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -160,10 +162,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const int s = i % STAGES, round = i / STAGES;
         if (round > 0 && !mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
         const uint32_t fb = full0 + 8 * s;
-        mbar_expect_tx(fb, A_BYTES + B_BYTES);
-        const uint32_t a_dst = tiles + s * (A_BYTES + B_BYTES);
+        mbar_expect_tx(fb, STAGE_BYTES);
+        const uint32_t a_dst = tiles + s * STAGE_BYTES;
         tma_load_2d(a_dst, &map_w, (kb0 + i) * BK, n0, fb);
-        tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);
+        tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);                 // hi part: columns [0, K)
+        tma_load_2d(a_dst + A_BYTES + B_BYTES, &map_x, K + (kb0 + i) * BK, m0, fb);   // lo part: columns [K, 2K)
         issued = i + 1;
       }
       if (*abort_flag) {
@@ -184,11 +187,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         ok = mbar_wait(full0 + 8 * s, round & 1, abort_flag, status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_addr = tiles + s * (A_BYTES + B_BYTES);
-        const uint64_t a_desc = smem_desc(a_addr), b_desc = smem_desc(a_addr + A_BYTES);
+        const uint32_t a_addr = tiles + s * STAGE_BYTES;
+        const uint64_t a_desc = smem_desc(a_addr), hi_desc = smem_desc(a_addr + A_BYTES),
+                       lo_desc = smem_desc(a_addr + A_BYTES + B_BYTES);
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k)     // 32 bytes further along K inside the swizzle row
-          umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+        for (int k = 0; k < BK / UMMA_K; ++k) {   // 32 bytes further along K inside the swizzle row
+          umma(tmem_base, a_desc + 2 * k, hi_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          umma(tmem_base, a_desc + 2 * k, lo_desc + 2 * k, idesc, 1u);
+        }
         umma_commit(empty0 + 8 * s);              // the stage is free once these MMAs have read it
       }
       if (ok) umma_commit(accum_bar);             // accumulator complete
@@ -213,7 +219,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               const float v = __uint_as_float(r[j]) + b;
               const size_t idx = (size_t)m * ldo + n;
               if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
-              else if (EPI == EPI_RELU_T) reinterpret_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(fmaxf(v, 0.f));
+              else if (EPI == EPI_RELU_T)      // the result is the next product's operand: row of 2N bf16, hi | lo
+                Operand<__nv_bfloat16>::store(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)m * ldo, N, n, fmaxf(v, 0.f));
               else atomicAdd(reinterpret_cast<float*>(out) + idx, v);
             }
           }
@@ -267,7 +274,7 @@ inline void tc_init(TcContext& c) {
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (major != 10) return;                       // tcgen05 exists on sm_100 only
   if (sms > 0) c.sm_count = sms;
-  if (!(tc_prepare_nb<16>() && tc_prepare_nb<32>() && tc_prepare_nb<64>() && tc_prepare_nb<128>() && tc_prepare_nb<256>())) {
+  if (!(tc_prepare_nb<16>() && tc_prepare_nb<32>() && tc_prepare_nb<64>() && tc_prepare_nb<128>())) {
     cudaGetLastError();
     return;
   }
@@ -309,11 +316,11 @@ inline bool tc_launch(cudaStream_t st, const CUtensorMap* mw, const CUtensorMap*
 // Returns true when the product was enqueued on the tensor-core path; false leaves it to the caller.
 inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const __nv_bfloat16* W, const __nv_bfloat16* bias,
                     int M, int N, int K, void* out, int ldo, int epi, int* status) {
-  if (!c.ready || K % 8 || M < 1 || N < 1) return false;
+  if (!c.ready || K % tc::BK || M < 1 || N < 1) return false;   // the hi and lo halves of a row are K apart: whole k-blocks only
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
-  const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+  const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
   const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
-  const CUtensorMap* mx = tc_map(c, X, M, K, nb);
+  const CUtensorMap* mx = tc_map(c, X, M, 2 * K, nb);
   if (!mw || !mx) return false;
   const int kb_total = (K + tc::BK - 1) / tc::BK;
   int splits = 1;
@@ -327,8 +334,7 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
     case 16: return tc_launch<16>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
     case 32: return tc_launch<32>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
     case 64: return tc_launch<64>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
-    case 128: return tc_launch<128>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
-    default: return tc_launch<256>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
+    default: return tc_launch<128>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
   }
 }
 template <typename T>

@@ -39,6 +39,28 @@ template <> struct Vec16<__nv_bfloat16> {
   }
 };
 
+// GEMM input operands.  In fp32 storage an operand row is K floats.  In bf16 storage it is
+// 2K bf16: columns [0,K) hold hi = bf16(v) and columns [K,2K) hold lo = bf16(v - hi), so the
+// tensor cores see v to ~16 mantissa bits (two bf16 products per element) while weights
+// and KV cache stay plain bf16.
+template <typename T> struct Operand;
+template <> struct Operand<float> {
+  static constexpr int PARTS = 1;
+  __device__ static __forceinline__ void store(float* row, int K, int c, float v) { row[c] = v; }
+  __device__ static __forceinline__ float load(const float* row, int K, int c) { return row[c]; }
+};
+template <> struct Operand<__nv_bfloat16> {
+  static constexpr int PARTS = 2;
+  __device__ static __forceinline__ void store(__nv_bfloat16* row, int K, int c, float v) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    row[c] = hi;
+    row[K + c] = __float2bfloat16_rn(v - __bfloat162float(hi));
+  }
+  __device__ static __forceinline__ float load(const __nv_bfloat16* row, int K, int c) {
+    return __bfloat162float(row[c]) + __bfloat162float(row[K + c]);
+  }
+};
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -94,7 +116,8 @@ __global__ void embed_pos_kernel(const int32_t* __restrict__ ids, const T* __res
 }
 
 // u[r, :] = (x[r, :] - mean) / sqrt(var + eps) * gamma + beta, biased variance, fp32 statistics.
-// Two passes over the row (mean, then centred second moment) for accuracy.
+// Two passes over the row (mean, then centred second moment) for accuracy.  u is a GEMM
+// operand (see Operand).
 template <typename T>
 __global__ void layernorm_kernel(const float* __restrict__ x, const T* __restrict__ gamma,
                                  const T* __restrict__ beta, T* __restrict__ u, int d, float eps,
@@ -108,9 +131,9 @@ __global__ void layernorm_kernel(const float* __restrict__ x, const T* __restric
   float q = 0.f;
   for (int c = threadIdx.x; c < d; c += blockDim.x) { const float t = xr[c] - mean; q += t * t; }
   const float rstd = rsqrtf(block_sum(q, red) / d + eps);
-  T* ur = u + (size_t)r * d;
+  T* ur = u + (size_t)r * d * Operand<T>::PARTS;
   for (int c = threadIdx.x; c < d; c += blockDim.x)
-    ur[c] = from_f32<T>((xr[c] - mean) * rstd * to_f32(gamma[c]) + to_f32(beta[c]));
+    Operand<T>::store(ur, d, c, (xr[c] - mean) * rstd * to_f32(gamma[c]) + to_f32(beta[c]));
 }
 
 // Writes this launch's keys and values into the layer's cache, in place:
@@ -279,7 +302,7 @@ __global__ void attn_combine_kernel(const float* __restrict__ part_acc, const fl
   for (int c = threadIdx.x; c < HD; c += blockDim.x) {
     float a = 0.f;
     for (int s = 0; s < n; ++s) a += part_acc[(slot0 + s) * HD + c] * exp2_safe(part_ml[(slot0 + s) * 2], M);
-    o[(size_t)r * H * HD + h * HD + c] = from_f32<T>(a * inv);
+    Operand<T>::store(o + (size_t)r * H * HD * Operand<T>::PARTS, H * HD, h * HD + c, a * inv);
   }
 }
 
@@ -319,7 +342,8 @@ __global__ void greedy_kernel(const float* __restrict__ logits, int vocab, int32
 
 // ---- CUDA-core GEMM -------------------------------------------------------------------
 // out[m, n] (+)= sum_k A[m, k] W[n, k] + bias[n], fp32 accumulation, 64x64 tile, 16-wide
-// k-steps, 256 threads with a 4x4 register tile each.
+// k-steps, 256 threads with a 4x4 register tile each.  A is an Operand row; the ReLU
+// epilogue writes an Operand row.
 enum : int { EPI_STORE_F32 = 0, EPI_RELU_T = 1, EPI_RESIDUAL_F32 = 2 };
 
 template <typename T, int EPI>
@@ -335,13 +359,13 @@ gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, int 
   const int lr = threadIdx.x >> 2;            // 0..63: tile row this thread loads
   const int lc = (threadIdx.x & 3) * 4;       // 0,4,8,12: first of its 4 k-columns
   const int am = m0 + lr, wn = n0 + lr;
-  const T* arow = am < M ? A + (size_t)am * lda : nullptr;
+  const T* arow = am < M ? A + (size_t)am * lda : nullptr;       // lda = K * Operand<T>::PARTS
   const T* wrow = wn < N ? W + (size_t)wn * ldw : nullptr;
   for (int k0 = 0; k0 < K; k0 += BK) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int k = k0 + lc + i;
-      As[lc + i][lr] = (arow && k < K) ? to_f32(arow[k]) : 0.f;
+      As[lc + i][lr] = (arow && k < K) ? Operand<T>::load(arow, K, k) : 0.f;
       Ws[lc + i][lr] = (wrow && k < K) ? to_f32(wrow[k]) : 0.f;
     }
     __syncthreads();
@@ -367,7 +391,7 @@ gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, int 
       if (n >= N) continue;
       const float v = acc[i][j] + (bias ? to_f32(bias[n]) : 0.f);
       if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[(size_t)m * ldo + n] = v;
-      else if (EPI == EPI_RELU_T) reinterpret_cast<T*>(out)[(size_t)m * ldo + n] = from_f32<T>(fmaxf(v, 0.f));
+      else if (EPI == EPI_RELU_T) Operand<T>::store(reinterpret_cast<T*>(out) + (size_t)m * ldo, N, n, fmaxf(v, 0.f));   // ldo = N * PARTS
       else reinterpret_cast<float*>(out)[(size_t)m * ldo + n] += v;
     }
   }

@@ -129,10 +129,10 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   A.rows_max = std::max(c.max_batch, chunk_rows);
   const size_t R = A.rows_max;
   A.x = take(R * d * 4);
-  A.u = take(R * d * e);
+  A.u = take(R * d * 4);                 // GEMM operands: K floats, or 2K bf16 (hi | lo), per row
   A.qkv = take(R * 3 * d * 4);
-  A.o = take(R * d * e);
-  A.y = take(R * (size_t)c.d_ffn * e);
+  A.o = take(R * d * 4);
+  A.y = take(R * (size_t)c.d_ffn * 4);
   const int maxT = c.max_prompt + c.max_gen;
   A.part_slots = std::max((size_t)c.max_batch * H * ((maxT + kMinChunk - 1) / kMinChunk), R * H);
   A.part_acc = take(A.part_slots * hd * 4);
@@ -183,12 +183,13 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, const T* bias, i
     done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status());
   if (!done) {
     dim3 grid((N + 63) / 64, (M + 63) / 64);
+    const int lda = K * sd::Operand<T>::PARTS;
     if (epi == sd::EPI_STORE_F32)
-      sd::gemm_simt_kernel<T, sd::EPI_STORE_F32><<<grid, 256, 0, h->stream>>>(A, K, W, K, bias, M, N, K, out, ldo);
+      sd::gemm_simt_kernel<T, sd::EPI_STORE_F32><<<grid, 256, 0, h->stream>>>(A, lda, W, K, bias, M, N, K, out, ldo);
     else if (epi == sd::EPI_RELU_T)
-      sd::gemm_simt_kernel<T, sd::EPI_RELU_T><<<grid, 256, 0, h->stream>>>(A, K, W, K, bias, M, N, K, out, ldo);
+      sd::gemm_simt_kernel<T, sd::EPI_RELU_T><<<grid, 256, 0, h->stream>>>(A, lda, W, K, bias, M, N, K, out, ldo);
     else
-      sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32><<<grid, 256, 0, h->stream>>>(A, K, W, K, bias, M, N, K, out, ldo);
+      sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32><<<grid, 256, 0, h->stream>>>(A, lda, W, K, bias, M, N, K, out, ldo);
   }
   Lc.end();
 }
@@ -249,7 +250,7 @@ void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int
   Lc.begin(SD_K_LAYERNORM);
   sd::layernorm_kernel<T><<<rows, ln_threads(d), 0, h->stream>>>(x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
-  launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f, sd::EPI_RELU_T);
+  launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f * sd::Operand<T>::PARTS, sd::EPI_RELU_T);
   launch_gemm<T>(Lc, SD_K_GEMM, y, (const T*)h->w_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
 }
 
