@@ -109,6 +109,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr) : "memory");
 }
 
+// Where the QKV epilogue puts its rows: features [0, d) are the query (fp32, into the qkv
+// buffer), [d, 2d) the key and [2d, 3d) the value, written straight into the layer's cache at
+// each token's position.  A 128-row tile never straddles two sections because d % 128 == 0.
+struct QkvOut {
+  __nv_bfloat16* Kc;
+  __nv_bfloat16* Vc;
+  int d, H, hd, cap;
+  RowMap map;
+};
+
 __host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
 __host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/; }
@@ -117,7 +127,7 @@ template <int NB, int EPI>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
-               int kb_per_split, int* __restrict__ status) {
+               int kb_per_split, int* __restrict__ status, const QkvOut qo) {
   constexpr int STAGES = stages_for(NB);
   constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
   constexpr int TMEM_COLS = NB < 32 ? 32 : NB;
@@ -219,6 +229,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               const float v = __uint_as_float(r[j]) + b;
               const size_t idx = (size_t)m * ldo + n;
               if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
+              else if (EPI == EPI_QKV_CACHE) {
+                if (n < qo.d) {
+                  reinterpret_cast<float*>(out)[idx] = v;
+                } else {
+                  int b, pos;
+                  qo.map.get(m, b, pos);
+                  const int cc = n < 2 * qo.d ? n - qo.d : n - 2 * qo.d;
+                  const int hh = cc / qo.hd, e = cc - hh * qo.hd;
+                  if (pos < qo.cap)
+                    (n < 2 * qo.d ? qo.Kc : qo.Vc)[(((size_t)b * qo.H + hh) * qo.cap + pos) * qo.hd + e] = __float2bfloat16_rn(v);
+                }
+              }
               else if (EPI == EPI_RELU_T)      // the result is the next product's operand: row of 2N bf16, hi | lo
                 Operand<__nv_bfloat16>::store(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)m * ldo, N, n, fmaxf(v, 0.f));
               else atomicAdd(reinterpret_cast<float*>(out) + idx, v);
@@ -256,7 +278,8 @@ inline bool tc_prepare() {
 }
 template <int NB>
 inline bool tc_prepare_nb() {
-  return tc_prepare<NB, EPI_STORE_F32>() && tc_prepare<NB, EPI_RELU_T>() && tc_prepare<NB, EPI_RESIDUAL_F32>();
+  return tc_prepare<NB, EPI_STORE_F32>() && tc_prepare<NB, EPI_RELU_T>() && tc_prepare<NB, EPI_RESIDUAL_F32>() &&
+         tc_prepare<NB, EPI_QKV_CACHE>();
 }
 
 inline void tc_init(TcContext& c) {
@@ -301,22 +324,26 @@ inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int co
 
 template <int NB>
 inline bool tc_launch(cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
-                      int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status) {
+                      int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status, const tc::QkvOut& qo) {
   dim3 grid((N + tc::BM - 1) / tc::BM, (M + NB - 1) / NB, splits);
   const int smem = tc::smem_bytes(NB);
   if (epi == EPI_STORE_F32)
-    tc::gemm_tc_kernel<NB, EPI_STORE_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status);
+    tc::gemm_tc_kernel<NB, EPI_STORE_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else if (epi == EPI_RELU_T)
-    tc::gemm_tc_kernel<NB, EPI_RELU_T><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status);
+    tc::gemm_tc_kernel<NB, EPI_RELU_T><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+  else if (epi == EPI_QKV_CACHE)
+    tc::gemm_tc_kernel<NB, EPI_QKV_CACHE><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else
-    tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status);
+    tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   return true;
 }
 
 // Returns true when the product was enqueued on the tensor-core path; false leaves it to the caller.
 inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const __nv_bfloat16* W, const __nv_bfloat16* bias,
-                    int M, int N, int K, void* out, int ldo, int epi, int* status) {
+                    int M, int N, int K, void* out, int ldo, int epi, int* status, const tc::QkvOut* qkv_out = nullptr) {
   if (!c.ready || K % tc::BK || M < 1 || N < 1) return false;   // the hi and lo halves of a row are K apart: whole k-blocks only
+  if (epi == EPI_QKV_CACHE && (!qkv_out || qkv_out->d % tc::BM || N != 3 * qkv_out->d)) return false;
+  const tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
   const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
   const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
@@ -331,14 +358,15 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   int kb_per_split = (kb_total + splits - 1) / splits;
   splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split
   switch (nb) {
-    case 16: return tc_launch<16>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
-    case 32: return tc_launch<32>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
-    case 64: return tc_launch<64>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
-    default: return tc_launch<128>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status);
+    case 16: return tc_launch<16>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 32: return tc_launch<32>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 64: return tc_launch<64>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    default: return tc_launch<128>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
   }
 }
 template <typename T>
-inline bool tc_gemm(TcContext&, cudaStream_t, const T*, const T*, const T*, int, int, int, void*, int, int, int*) {
+inline bool tc_gemm(TcContext&, cudaStream_t, const T*, const T*, const T*, int, int, int, void*, int, int, int*,
+                    const tc::QkvOut* = nullptr) {
   return false;                                  // fp32 storage runs on the CUDA-core kernel
 }
 

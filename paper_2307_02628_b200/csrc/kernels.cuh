@@ -344,7 +344,7 @@ __global__ void greedy_kernel(const float* __restrict__ logits, int vocab, int32
 // out[m, n] (+)= sum_k A[m, k] W[n, k] + bias[n], fp32 accumulation, 64x64 tile, 16-wide
 // k-steps, 256 threads with a 4x4 register tile each.  A is an Operand row; the ReLU
 // epilogue writes an Operand row.
-enum : int { EPI_STORE_F32 = 0, EPI_RELU_T = 1, EPI_RESIDUAL_F32 = 2 };
+enum : int { EPI_STORE_F32 = 0, EPI_RELU_T = 1, EPI_RESIDUAL_F32 = 2, EPI_QKV_CACHE = 3 /* tensor-core kernel only */ };
 
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256)

@@ -166,6 +166,11 @@ struct Launcher {
     cudaEventRecord(t.a, h->stream);
     h->timed.push_back(t);
   }
+  void cancel() {          // begin() was called but nothing was launched
+    if (!timing) return;
+    cudaEventDestroy(h->timed.back().a); cudaEventDestroy(h->timed.back().b);
+    h->timed.pop_back();
+  }
   void end() {
     ++count;
     if (cudaGetLastError() != cudaSuccess) err = SD_ERR_CUDA;
@@ -192,6 +197,22 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, const T* bias, i
       sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32><<<grid, 256, 0, h->stream>>>(A, lda, W, K, bias, M, N, K, out, ldo);
   }
   Lc.end();
+}
+
+// QKV projection with the K/V rows written straight into the cache by the GEMM epilogue
+// (tensor-core path only).  Returns false when that path does not take the product.
+template <typename T>
+bool launch_qkv_to_cache(Launcher&, const T*, const T*, const T*, int, int, float*, T*, T*, int, sd::RowMap) { return false; }
+template <>
+bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, const bf16* bias, int rows, int d, float* qkv,
+                               bf16* Kc, bf16* Vc, int cap, sd::RowMap map) {
+  sd_handle* h = Lc.h;
+  if (h->opt_gemm == 1) return false;
+  const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map};
+  Lc.begin(SD_K_GEMM);
+  const bool done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
+  if (done) Lc.end(); else Lc.cancel();
+  return done;
 }
 
 template <typename T, int HD>
@@ -241,10 +262,12 @@ void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int
   Lc.begin(SD_K_LAYERNORM);
   sd::layernorm_kernel<T><<<rows, ln_threads(d), 0, h->stream>>>(x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
-  launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
-  Lc.begin(SD_K_KV_APPEND);
-  sd::kv_append_kernel<T><<<rows, 256, 0, h->stream>>>(qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
-  Lc.end();
+  if (!launch_qkv_to_cache<T>(Lc, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, d, qkv, Kc, Vc, cap, map)) {
+    launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
+    Lc.begin(SD_K_KV_APPEND);
+    sd::kv_append_kernel<T><<<rows, 256, 0, h->stream>>>(qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
+    Lc.end();
+  }
   launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
   launch_gemm<T>(Lc, SD_K_GEMM, o, (const T*)h->w_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
   Lc.begin(SD_K_LAYERNORM);
