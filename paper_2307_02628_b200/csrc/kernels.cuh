@@ -1,5 +1,5 @@
 // CUDA-core kernels of the skip-decode step: embedding, LayerNorm, KV append,
-// split-KV decode attention and its combine, greedy argmax, and the CUDA-core GEMM
+// split-KV decode attention (with its merge), greedy argmax, and the CUDA-core GEMM
 // used by the fp32 configuration (and as the fallback for shapes the tensor-core
 // GEMM does not take).  T is the storage type: float or __nv_bfloat16.
 #pragma once
@@ -160,8 +160,12 @@ __global__ void kv_append_kernel(const float* __restrict__ qkv, T* __restrict__ 
 // LPK = HD / VEC lanes owns one key at a time: each lane holds VEC consecutive dims (one
 // 16-byte load of K and of V), the dot product is finished with xor-shuffles inside the
 // group, and every group runs its own online softmax in base 2.  Groups are merged by
-// shuffles inside a warp and through shared memory across warps.  Output per (row, head,
-// chunk): unnormalised accumulator[HD], running max m (base-2 exponent) and sum l.
+// shuffles inside a warp and through shared memory across warps.  With one chunk the block
+// writes the attention output o[r, h*HD + c] (a GEMM operand) itself; with several, every
+// block stores (unnormalised accumulator[HD], running max m as a base-2 exponent, sum l) and
+// the block that arrives last at a per-(row, head) counter merges them:
+// o = sum_s acc_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).  Partials written by other SMs are read
+// with L2 loads (the buffers are reused every layer, so L1 could hold stale lines).
 __device__ __forceinline__ float exp2_safe(float a, float m) {   // 2^(a - m), 0 when a = -inf
   return a == -INFINITY ? 0.f : exp2f(a - m);
 }
@@ -170,7 +174,7 @@ template <typename T, int HD, int UNROLL>
 __global__ void __launch_bounds__(128)
 attn_partial_kernel(const float* __restrict__ qkv, int ldq, const T* __restrict__ Kc, const T* __restrict__ Vc,
                     int cap, int H, RowMap map, int chunk, int max_chunks,
-                    float* __restrict__ part_acc, float* __restrict__ part_ml) {
+                    float* part_acc, float* part_ml, int* __restrict__ counters, T* __restrict__ o) {
   constexpr int VEC = Vec16<T>::N;
   constexpr int LPK = HD / VEC;              // lanes per key
   constexpr int KPW = 32 / LPK;              // keys per warp step
@@ -259,16 +263,33 @@ attn_partial_kernel(const float* __restrict__ qkv, int ldq, const T* __restrict_
   // merge the warps
   __shared__ float sm_acc[NW][HD];
   __shared__ float sm_m[NW], sm_l[NW];
+  __shared__ int sm_last;
   if (grp == 0) {
 #pragma unroll
     for (int v = 0; v < VEC; ++v) sm_acc[warp][sub * VEC + v] = acc[v];
     if (sub == 0) { sm_m[warp] = m; sm_l[warp] = l; }
   }
   __syncthreads();
-  const size_t slot = (size_t)rh * max_chunks + blockIdx.y;
   float M = sm_m[0];
 #pragma unroll
   for (int w = 1; w < NW; ++w) M = fmaxf(M, sm_m[w]);
+  float L = 0.f;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) L += sm_l[w] * exp2_safe(sm_m[w], M);
+  const int n_valid = (T_len + chunk - 1) / chunk;          // chunks of this (row, head) that hold keys
+  T* orow = o + (size_t)r * H * HD * Operand<T>::PARTS;
+  if (n_valid == 1) {                                       // the only chunk: normalise and finish here
+    const float inv = 1.f / L;
+    for (int c = threadIdx.x; c < HD; c += blockDim.x) {
+      float a = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) a += sm_acc[w][c] * exp2_safe(sm_m[w], M);
+      Operand<T>::store(orow, H * HD, h * HD + c, a * inv);
+    }
+    return;
+  }
+  const size_t slot0 = (size_t)rh * max_chunks;
+  const size_t slot = slot0 + blockIdx.y;
   for (int c = threadIdx.x; c < HD; c += blockDim.x) {
     float a = 0.f;
 #pragma unroll
@@ -276,33 +297,32 @@ attn_partial_kernel(const float* __restrict__ qkv, int ldq, const T* __restrict_
     part_acc[slot * HD + c] = a;
   }
   if (threadIdx.x == 0) {
-    float L = 0.f;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) L += sm_l[w] * exp2_safe(sm_m[w], M);
     part_ml[slot * 2] = M;
     part_ml[slot * 2 + 1] = L;
   }
-}
-
-// o[r, h*HD + c] = sum_s acc_s[c] 2^(m_s - M) / sum_s l_s 2^(m_s - M) over the chunks that hold keys.
-template <typename T, int HD>
-__global__ void attn_combine_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
-                                    T* __restrict__ o, int H, int cap, RowMap map, int chunk, int max_chunks) {
-  const int rh = blockIdx.x, r = rh / H, h = rh - r * H;
-  int b, pos;
-  map.get(r, b, pos);
-  const int T_len = min(pos + 1, cap);
-  const int n = min((T_len + chunk - 1) / chunk, max_chunks);
-  const size_t slot0 = (size_t)rh * max_chunks;
-  float M = -INFINITY;
-  for (int s = 0; s < n; ++s) M = fmaxf(M, part_ml[(slot0 + s) * 2]);
-  float L = 0.f;
-  for (int s = 0; s < n; ++s) L += part_ml[(slot0 + s) * 2 + 1] * exp2_safe(part_ml[(slot0 + s) * 2], M);
-  const float inv = 1.f / L;
+  // The block that finishes last for this (row, head) merges all chunks.  Nobody waits: each
+  // block publishes its partial, bumps the counter and leaves; only the last one goes on.
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int done = atomicAdd(&counters[rh], 1);
+    sm_last = (done == n_valid - 1);
+    if (sm_last) counters[rh] = 0;                          // ready for the next launch
+  }
+  __syncthreads();
+  if (!sm_last) return;
+  __threadfence();
+  float Mg = -INFINITY;
+  for (int s = 0; s < n_valid; ++s) Mg = fmaxf(Mg, __ldcg(part_ml + (slot0 + s) * 2));
+  float Lg = 0.f;
+  for (int s = 0; s < n_valid; ++s)
+    Lg += __ldcg(part_ml + (slot0 + s) * 2 + 1) * exp2_safe(__ldcg(part_ml + (slot0 + s) * 2), Mg);
+  const float inv = 1.f / Lg;
   for (int c = threadIdx.x; c < HD; c += blockDim.x) {
     float a = 0.f;
-    for (int s = 0; s < n; ++s) a += part_acc[(slot0 + s) * HD + c] * exp2_safe(part_ml[(slot0 + s) * 2], M);
-    Operand<T>::store(o + (size_t)r * H * HD * Operand<T>::PARTS, H * HD, h * HD + c, a * inv);
+    for (int s = 0; s < n_valid; ++s)
+      a += __ldcg(part_acc + (slot0 + s) * HD + c) * exp2_safe(__ldcg(part_ml + (slot0 + s) * 2), Mg);
+    Operand<T>::store(orow, H * HD, h * HD + c, a * inv);
   }
 }
 

@@ -28,7 +28,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Arena {            // byte offsets into the caller's arena
   std::vector<size_t> k_off, v_off;
   std::vector<int> cap;
-  size_t x, u, qkv, o, y, part_acc, part_ml, row_index, ids, logits, scalars, total;
+  size_t x, u, qkv, o, y, part_acc, part_ml, counters, row_index, ids, logits, scalars, total;
   int rows_max;
   size_t part_slots;
 };
@@ -137,6 +137,7 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   A.part_slots = std::max((size_t)c.max_batch * H * ((maxT + kMinChunk - 1) / kMinChunk), R * H);
   A.part_acc = take(A.part_slots * hd * 4);
   A.part_ml = take(A.part_slots * 2 * 4);
+  A.counters = take(R * H * 4);          // split-KV arrival counters, one per (row, head); zero between launches
   A.row_index = take((size_t)c.max_batch * 4);
   A.ids = take((size_t)c.max_batch * 4);
   A.logits = take((size_t)c.max_batch * c.vocab * 4);
@@ -223,11 +224,8 @@ void launch_attention_hd(Launcher& Lc, const T* Kc, const T* Vc, int cap, int ro
   Lc.begin(SD_K_ATTENTION);
   dim3 grid(rows * H, n_chunks);
   sd::attn_partial_kernel<T, HD, 4><<<grid, 128, 0, h->stream>>>(
-      h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml);
-  Lc.end();
-  Lc.begin(SD_K_COMBINE);
-  sd::attn_combine_kernel<T, HD><<<rows * H, HD < 64 ? 32 : 64, 0, h->stream>>>(
-      Lc.part_acc, Lc.part_ml, h->at<T>(h->A.o), H, cap, map, chunk, n_chunks);
+      h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml,
+      h->at<int>(h->A.counters), h->at<T>(h->A.o));
   Lc.end();
 }
 
@@ -467,7 +465,10 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
   h->lm_head = w->lm_head ? w->lm_head : w->tok_emb;
   h->arena = static_cast<char*>(arena);
   h->stream = static_cast<cudaStream_t>(stream);
-  if (cudaMemsetAsync(h->arena + h->A.scalars, 0, 256, h->stream) != cudaSuccess) { cudaGetLastError(); delete h; return SD_ERR_CUDA; }
+  if (cudaMemsetAsync(h->arena + h->A.scalars, 0, 256, h->stream) != cudaSuccess ||
+      cudaMemsetAsync(h->arena + h->A.counters, 0, (size_t)h->A.rows_max * cfg->n_heads * 4, h->stream) != cudaSuccess) {
+    cudaGetLastError(); delete h; return SD_ERR_CUDA;
+  }
   sd::tc_init(h->tc);
   *out = h;
   return SD_OK;
@@ -563,8 +564,8 @@ int sd_decode_step_static(sd_handle* h, const int32_t* d_ids, int position, floa
   float* part_acc = static_cast<float*>(base);
   float* part_ml = reinterpret_cast<float*>(static_cast<char*>(base) + acc_bytes);
   int64_t launched = 0;
-  // every partial slot the combine kernel reads is written by the attention kernel of the same
-  // layer first, so nothing in the array has to start at zero
+  // every partial slot the merging block reads was written earlier in the same attention launch,
+  // so nothing in the array has to start at zero
   const int err = h->cfg.dtype == SD_DTYPE_BF16
       ? enqueue_decode<bf16>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, false, &launched, part_acc, part_ml)
       : enqueue_decode<float>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, false, &launched, part_acc, part_ml);
