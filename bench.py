@@ -208,10 +208,12 @@ def gpu_arm(args, wl, rank, world):
             dist.barrier()
         torch.cuda.synchronize(device)
 
+    G_run = G if args.max_gen_steps <= 0 else min(G, args.max_gen_steps)   # < G only for profiler runs
+
     def one_pass():
         dec.rewind()
         dec.greedy(logits0, ids)
-        for g in range(G):
+        for g in range(G_run):
             dec.decode_step(ids, P + g, logits)
             dec.greedy(logits, ids)
 
@@ -253,16 +255,18 @@ def gpu_arm(args, wl, rank, world):
 
         def e2e_pass():
             dec.rewind()
-            for g in range(G):
+            for g in range(G_run):
                 dec.decode_step_host(h_ids[g], P + g, h_logits)
 
-        e2e_pass()
-        barrier()
-        te = time.perf_counter()
-        for _ in range(args.e2e_steps):
+        e2e_s = float("nan")
+        if args.e2e_steps > 0:
             e2e_pass()
-        barrier()
-        e2e_s = (time.perf_counter() - te) / args.e2e_steps
+            barrier()
+            te = time.perf_counter()
+            for _ in range(args.e2e_steps):
+                e2e_pass()
+            barrier()
+            e2e_s = (time.perf_counter() - te) / args.e2e_steps
         if dist is not None:
             t = torch.tensor([e2e_s], device=device)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -274,7 +278,7 @@ def gpu_arm(args, wl, rank, world):
         dec.greedy(logits0, ids)
         attn_bytes = 0.0
         e = 4 if s.dtype == "fp32" else 2
-        for g in range(G):
+        for g in range(G_run if args.profile_every > 0 else 0):
             sampled = (g % args.profile_every == 0)
             dec.set_option(binding.SD_OPT_TIMING, 1 if sampled else 0)
             dec.decode_step(ids, P + g, logits)
@@ -290,21 +294,21 @@ def gpu_arm(args, wl, rank, world):
             dec.schedule(s.n_layers, s.n_layers, 0, G)
             one_pass()
             ms_full = timed(one_pass, max(1, min(2, args.steps)))
-            full = {"ms_per_step": ms_full, "tokens_per_s": world * B * G / (ms_full / 1e3),
+            full = {"ms_per_step": ms_full, "tokens_per_s": world * B * G_run / (ms_full / 1e3),
                     "speedup_skip_over_full": ms_full / ms_step,
-                    "byte_model_bound": step_bytes(wl, [s.n_layers] * G) / step_bytes(wl, n_active)}
+                    "byte_model_bound": step_bytes(wl, [s.n_layers] * G_run) / step_bytes(wl, n_active[:G_run])}
 
     peak, peak_kind = measured_peaks()
-    value = world * B * G / (ms_step / 1e3)
-    total_bytes = step_bytes(wl, n_active)
+    value = world * B * G_run / (ms_step / 1e3)
+    total_bytes = step_bytes(wl, n_active[:G_run])
     achieved = attn_bytes / (attn_ms / 1e3) / 1e9 if attn_ms > 0 else None
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic", "config": bench_config(wl, args),
         "clocks": clock_info, "gpu_launches": int(launches),
-        "e2e": {"value": world * B * G / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": G * B * 4,
-                "d2h_bytes_per_step": G * B * s.vocab * 4},
+        "e2e": {"value": world * B * G_run / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": G_run * B * 4,
+                "d2h_bytes_per_step": G_run * B * s.vocab * 4},
         "roofline": {"kernel": "attn_partial_kernel (split-KV decode attention)", "bound": "hbm", "achieved": achieved,
                      "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
                      "traffic": None, "launches_timed": int(attn_n),
@@ -316,6 +320,8 @@ def gpu_arm(args, wl, rank, world):
         "full_layer": full, "prefill_s": t_prefill, "weights_s": t_weights,
         "mean_active_layers": sum(n_active) / len(n_active),
     }
+    if G_run != G:
+        line["partial_pass"] = f"first {G_run} of {G} decode steps per pass: a profiler run, not a benchmark value"
     dec.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = torch.get_num_threads()
@@ -337,6 +343,8 @@ def main():
     ap.add_argument("--config", default="c4", choices=sorted(synth.CONFIGS))
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--profile-every", type=int, default=8)
+    ap.add_argument("--max-gen-steps", type=int, default=0,
+                    help="run only the first N decode steps of each pass (for short profiler captures)")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-rows", type=int, default=1)

@@ -353,7 +353,7 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   int splits = 1;
   if (epi == EPI_RESIDUAL_F32) {                 // partial sums may be added in any order
     const int tiles = ((N + tc::BM - 1) / tc::BM) * ((M + nb - 1) / nb);
-    splits = std::max(1, std::min(kb_total / 4, (c.sm_count + tiles - 1) / tiles));
+    splits = std::max(1, std::min(kb_total / 4, c.sm_count / tiles));     // one wave: never more blocks than SMs
   }
   int kb_per_split = (kb_total + splits - 1) / splits;
   splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split
