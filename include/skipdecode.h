@@ -203,7 +203,8 @@ enum {
   SD_OPT_GRAPHS = 1,       /* 1 (default): replay one CUDA graph per step shape; 0: plain launches */
   SD_OPT_ATTN_CHUNK = 2,   /* keys per split of the decode attention (multiple of 32); 0 = automatic */
   SD_OPT_GEMM = 3,         /* 0 = automatic; 1 = CUDA-core GEMMs only (bf16 mode as well)          */
-  SD_OPT_TIMING = 4        /* 1: record per-kernel-class device time (plain launches, slower)      */
+  SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
+  SD_OPT_PDL = 5           /* 1 (default): programmatic dependent launch between the step's kernels */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 

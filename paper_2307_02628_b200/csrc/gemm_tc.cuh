@@ -162,22 +162,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
-      int issued = 0;
+      // The weights do not depend on the previous kernel: start streaming the first stages'
+      // W tiles while it is still finishing, and only then wait for it before touching X.
+      const int early = nkb < STAGES ? nkb : STAGES;
+      for (int i = 0; i < early; ++i) {
+        const uint32_t fb = full0 + 8 * i;
+        mbar_expect_tx(fb, STAGE_BYTES);
+        tma_load_2d(tiles + i * STAGE_BYTES, &map_w, (kb0 + i) * BK, n0, fb);
+      }
+      pdl_wait();
+      int issued = early;
       for (int i = 0; i < nkb; ++i) {
         const int s = i % STAGES, round = i / STAGES;
-        if (round > 0 && !mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
         const uint32_t fb = full0 + 8 * s;
-        mbar_expect_tx(fb, STAGE_BYTES);
         const uint32_t a_dst = tiles + s * STAGE_BYTES;
-        tma_load_2d(a_dst, &map_w, (kb0 + i) * BK, n0, fb);
+        if (round > 0) {
+          if (!mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
+          mbar_expect_tx(fb, STAGE_BYTES);
+          tma_load_2d(a_dst, &map_w, (kb0 + i) * BK, n0, fb);
+        }
         tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);                 // hi part: columns [0, K)
         tma_load_2d(a_dst + A_BYTES + B_BYTES, &map_x, K + (kb0 + i) * BK, m0, fb);   // lo part: columns [K, 2K)
-        issued = i + 1;
+        if (i + 1 > issued) issued = i + 1;
       }
       if (*abort_flag) {
         // drain: wait (bounded) until every copy issued has landed before the CTA exits
@@ -210,6 +222,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       if (ok) umma_commit(accum_bar);             // accumulator complete
     }
   } else {
+    pdl_wait();                                   // bias aside, the epilogue reads and writes buffers earlier kernels own
     const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, +32) belong to this warp
     const int n = n0 + quarter * 32 + lane;
     if (mbar_wait(accum_bar, 0, abort_flag, status)) {
@@ -268,6 +281,7 @@ struct TcContext {
   EncodeTiledFn encode = nullptr;
   int ready = 0;
   int sm_count = 148;
+  bool pdl = false;      // launch with the programmatic-dependent-launch attribute
   // (pointer, rows, cols, box rows) -> tensor map of a row-major bf16 matrix, 64-column boxes, 128-byte swizzle
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
 };
@@ -323,18 +337,18 @@ inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int co
 }
 
 template <int NB>
-inline bool tc_launch(cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
+inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
                       int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status, const tc::QkvOut& qo) {
   dim3 grid((N + tc::BM - 1) / tc::BM, (M + NB - 1) / NB, splits);
   const int smem = tc::smem_bytes(NB);
   if (epi == EPI_STORE_F32)
-    tc::gemm_tc_kernel<NB, EPI_STORE_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_STORE_F32>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else if (epi == EPI_RELU_T)
-    tc::gemm_tc_kernel<NB, EPI_RELU_T><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RELU_T>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else if (epi == EPI_QKV_CACHE)
-    tc::gemm_tc_kernel<NB, EPI_QKV_CACHE><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_QKV_CACHE>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else
-    tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32><<<grid, 192, smem, st>>>(*mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   return true;
 }
 
@@ -358,10 +372,10 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   int kb_per_split = (kb_total + splits - 1) / splits;
   splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split
   switch (nb) {
-    case 16: return tc_launch<16>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    case 32: return tc_launch<32>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    case 64: return tc_launch<64>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    default: return tc_launch<128>(st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 16: return tc_launch<16>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 32: return tc_launch<32>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 64: return tc_launch<64>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    default: return tc_launch<128>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
   }
 }
 template <typename T>

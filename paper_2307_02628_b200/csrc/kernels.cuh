@@ -11,6 +11,14 @@ namespace sd {
 
 enum : int { STATUS_BAD_TOKEN = 1, STATUS_WAIT_EXPIRED = 2, STATUS_BAD_SHAPE = 4 };
 
+// Programmatic dependent launch.  Every kernel of the step calls pdl_begin() before it touches
+// anything an earlier kernel wrote: it lets the next kernel in the stream start its own
+// prologue early and then blocks until the previous kernel has completed and its writes are
+// visible.  Both instructions do nothing when the launch carries no programmatic attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_begin() { pdl_launch_dependents(); pdl_wait(); }
+
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T from_f32(float v);
@@ -100,6 +108,7 @@ template <typename T>
 __global__ void embed_pos_kernel(const int32_t* __restrict__ ids, const T* __restrict__ tok_emb,
                                  const T* __restrict__ pos_emb, float* __restrict__ x, int d, int vocab,
                                  int max_pos, RowMap map, int* __restrict__ status) {
+  pdl_begin();
   const int r = blockIdx.x;
   int b, pos;
   map.get(r, b, pos);
@@ -123,6 +132,7 @@ __global__ void layernorm_kernel(const float* __restrict__ x, const T* __restric
                                  const T* __restrict__ beta, T* __restrict__ u, int d, float eps,
                                  const int* __restrict__ row_index) {
   __shared__ float red[33];
+  pdl_begin();
   const int r = blockIdx.x;
   const float* xr = x + (size_t)(row_index ? row_index[r] : r) * d;
   float s = 0.f;
@@ -142,6 +152,7 @@ __global__ void layernorm_kernel(const float* __restrict__ x, const T* __restric
 template <typename T>
 __global__ void kv_append_kernel(const float* __restrict__ qkv, T* __restrict__ Kc, T* __restrict__ Vc,
                                  int d, int H, int hd, int cap, RowMap map) {
+  pdl_begin();
   const int r = blockIdx.x;
   int b, pos;
   map.get(r, b, pos);
@@ -182,6 +193,7 @@ attn_partial_kernel(const float* __restrict__ qkv, int ldq, const T* __restrict_
   constexpr int G = NW * KPW;                // key groups per block
   static_assert(LPK >= 1 && LPK <= 32 && (LPK & (LPK - 1)) == 0, "head_dim / vector width must be a power of two <= 32");
 
+  pdl_begin();
   const int rh = blockIdx.x, r = rh / H, h = rh - r * H;
   int b, pos;
   map.get(r, b, pos);
@@ -326,6 +338,20 @@ attn_partial_kernel(const float* __restrict__ qkv, int ldq, const T* __restrict_
   }
 }
 
+// Host side: launch with the programmatic-dependent-launch attribute when `pdl` is set.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(bool pdl, cudaStream_t stream, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // next[b] = lowest index of the maximum of logits[b, :]
 __global__ void greedy_kernel(const float* __restrict__ logits, int vocab, int32_t* __restrict__ next) {
   __shared__ float sv[32];
@@ -371,6 +397,7 @@ __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, int ldw,
                  const T* __restrict__ bias, int M, int N, int K, void* __restrict__ out, int ldo) {
   constexpr int BM = 64, BN = 64, BK = 16;
+  pdl_begin();
   __shared__ float As[BK][BM + 4];
   __shared__ float Ws[BK][BN + 4];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;

@@ -53,7 +53,7 @@ struct sd_handle {
   int B = 0, P = 0, next_pos = 0;
   int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
-  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0;
+  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = 1;
   // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
   struct Graph { cudaGraphExec_t exec; int64_t nodes; };
   std::map<std::tuple<int, int, int, int, int, const void*, const void*>, Graph> graphs;
@@ -191,11 +191,11 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, const T* bias, i
     dim3 grid((N + 63) / 64, (M + 63) / 64);
     const int lda = K * sd::Operand<T>::PARTS;
     if (epi == sd::EPI_STORE_F32)
-      sd::gemm_simt_kernel<T, sd::EPI_STORE_F32><<<grid, 256, 0, h->stream>>>(A, lda, W, K, bias, M, N, K, out, ldo);
+      sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::gemm_simt_kernel<T, sd::EPI_STORE_F32>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
     else if (epi == sd::EPI_RELU_T)
-      sd::gemm_simt_kernel<T, sd::EPI_RELU_T><<<grid, 256, 0, h->stream>>>(A, lda, W, K, bias, M, N, K, out, ldo);
+      sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::gemm_simt_kernel<T, sd::EPI_RELU_T>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
     else
-      sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32><<<grid, 256, 0, h->stream>>>(A, lda, W, K, bias, M, N, K, out, ldo);
+      sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
   }
   Lc.end();
 }
@@ -223,8 +223,7 @@ void launch_attention_hd(Launcher& Lc, const T* Kc, const T* Vc, int cap, int ro
   const int H = h->cfg.n_heads;
   Lc.begin(SD_K_ATTENTION);
   dim3 grid(rows * H, n_chunks);
-  sd::attn_partial_kernel<T, HD, 4><<<grid, 128, 0, h->stream>>>(
-      h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml,
+  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::attn_partial_kernel<T, HD, 4>, dim3(grid), dim3(128), 0, h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml,
       h->at<int>(h->A.counters), h->at<T>(h->A.o));
   Lc.end();
 }
@@ -258,18 +257,18 @@ void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int
   const int cap = h->A.cap[l];
 
   Lc.begin(SD_K_LAYERNORM);
-  sd::layernorm_kernel<T><<<rows, ln_threads(d), 0, h->stream>>>(x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
+  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
   if (!launch_qkv_to_cache<T>(Lc, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, d, qkv, Kc, Vc, cap, map)) {
     launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
     Lc.begin(SD_K_KV_APPEND);
-    sd::kv_append_kernel<T><<<rows, 256, 0, h->stream>>>(qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
+    sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::kv_append_kernel<T>, dim3(rows), dim3(256), 0, qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
     Lc.end();
   }
   launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
   launch_gemm<T>(Lc, SD_K_GEMM, o, (const T*)h->w_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
   Lc.begin(SD_K_LAYERNORM);
-  sd::layernorm_kernel<T><<<rows, ln_threads(d), 0, h->stream>>>(x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
+  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
   launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f * sd::Operand<T>::PARTS, sd::EPI_RELU_T);
   launch_gemm<T>(Lc, SD_K_GEMM, y, (const T*)h->w_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
@@ -279,7 +278,7 @@ template <typename T>
 void enqueue_embed(Launcher& Lc, const int32_t* ids, int rows, sd::RowMap map) {
   sd_handle* h = Lc.h;
   Lc.begin(SD_K_EMBED);
-  sd::embed_pos_kernel<T><<<rows, 256, 0, h->stream>>>(ids, (const T*)h->tok_emb, (const T*)h->pos_emb, h->at<float>(h->A.x),
+  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::embed_pos_kernel<T>, dim3(rows), dim3(256), 0, ids, (const T*)h->tok_emb, (const T*)h->pos_emb, h->at<float>(h->A.x),
                                                       h->cfg.d_model, h->cfg.vocab, h->cfg.max_pos, map, h->status());
   Lc.end();
 }
@@ -290,7 +289,7 @@ void enqueue_head(Launcher& Lc, int rows, const int* row_index, float* d_logits)
   sd_handle* h = Lc.h;
   const sd_config& c = h->cfg;
   Lc.begin(SD_K_LAYERNORM);
-  sd::layernorm_kernel<T><<<rows, ln_threads(c.d_model), 0, h->stream>>>(h->at<float>(h->A.x), (const T*)h->lnf_g, (const T*)h->lnf_b,
+  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(c.d_model)), 0, h->at<float>(h->A.x), (const T*)h->lnf_g, (const T*)h->lnf_b,
                                                                         h->at<T>(h->A.u), c.d_model, c.ln_eps, row_index);
   Lc.end();
   launch_gemm<T>(Lc, SD_K_LM_HEAD, h->at<T>(h->A.u), (const T*)h->lm_head, (const T*)nullptr, rows, c.vocab, c.d_model,
@@ -470,6 +469,7 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
     cudaGetLastError(); delete h; return SD_ERR_CUDA;
   }
   sd::tc_init(h->tc);
+  h->tc.pdl = h->opt_pdl != 0;
   *out = h;
   return SD_OK;
 }
@@ -624,6 +624,9 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value < 0 || value > 1) return SD_ERR_ARG;
       if (value != h->opt_gemm) drop_graphs(h);
       h->opt_gemm = value; return SD_OK;
+    case SD_OPT_PDL:
+      if ((value != 0) != (h->opt_pdl != 0)) drop_graphs(h);
+      h->opt_pdl = value ? 1 : 0; h->tc.pdl = h->opt_pdl != 0; return SD_OK;
     case SD_OPT_TIMING:
       if (h->opt_timing && !value) collect_timing(h);
       h->opt_timing = value ? 1 : 0; return SD_OK;

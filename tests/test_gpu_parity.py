@@ -218,3 +218,28 @@ def test_tensor_core_and_cuda_core_gemm_paths_agree(B, P):
     # same bf16 operands, fp32 accumulation in a different order
     # a different summation order flips some bf16 roundings of the activations: ulp-scale differences
     assert float((outs[0] - outs[1]).abs().max()) < 1e-2
+
+
+def test_launch_modes_compute_the_same_function():
+    """CUDA graphs and programmatic dependent launch only change how kernels are enqueued."""
+    from paper_2307_02628_b200 import binding
+    runs = {}
+    for shape in (synth.TINY, synth.ModelShape("modes-bf16", 3, 256, 2, 512, 640, 160, "bf16")):
+        wl = synth.Workload(shape, 5, 40, 24, 3, 2, 1)
+        w = synth.make_weights(shape, seed=9)
+        prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+        ref = harness.oracle_run_forced(wl, w, prompts, forced)
+        for graphs in (1, 0):
+            for pdl in (1, 0):
+                dec = harness.make_decoder(wl, w)
+                dec.set_option(binding.SD_OPT_GRAPHS, graphs)
+                dec.set_option(binding.SD_OPT_PDL, pdl)
+                out = harness.gpu_run_forced(dec, wl, prompts, forced)
+                dec.close()
+                _check(out, ref, shape.dtype, f"{shape.name} graphs={graphs} pdl={pdl}")
+                runs[(shape.name, graphs, pdl)] = out
+        if shape.dtype == "fp32":            # no atomics on this path: bit-identical in every mode
+            base = runs[(shape.name, 1, 1)]
+            for key, out in runs.items():
+                if key[0] == shape.name:
+                    assert torch.equal(out, base), key
