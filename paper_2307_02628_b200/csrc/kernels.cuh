@@ -128,20 +128,56 @@ __global__ void embed_pos_kernel(const int32_t* __restrict__ ids, const T* __res
 // Two passes over the row (mean, then centred second moment) for accuracy.  u is a GEMM
 // operand (see Operand).
 template <typename T>
-__global__ void layernorm_kernel(const float* __restrict__ x, const T* __restrict__ gamma,
-                                 const T* __restrict__ beta, T* __restrict__ u, int d, float eps,
-                                 const int* __restrict__ row_index) {
+__global__ void __launch_bounds__(256)
+layernorm_kernel(const float* __restrict__ x, const T* __restrict__ gamma, const T* __restrict__ beta,
+                 T* __restrict__ u, int d, float eps, const int* __restrict__ row_index) {
+  constexpr int MAXV = 4;                       // float4 vectors a thread keeps in registers
   __shared__ float red[33];
   pdl_begin();
   const int r = blockIdx.x;
   const float* xr = x + (size_t)(row_index ? row_index[r] : r) * d;
+  T* ur = u + (size_t)r * d * Operand<T>::PARTS;
+  const int nvec = d >> 2;                      // d is a multiple of 8
+  if (nvec <= MAXV * (int)blockDim.x) {         // the row fits in registers: one read of x
+    float4 v[MAXV];
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const int k = i * blockDim.x + threadIdx.x;
+      v[i] = k < nvec ? reinterpret_cast<const float4*>(xr)[k] : make_float4(0.f, 0.f, 0.f, 0.f);
+      s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+    }
+    const float mean = block_sum(s, red) / d;
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const int k = i * blockDim.x + threadIdx.x;
+      if (k < nvec) {
+        const float a = v[i].x - mean, b = v[i].y - mean, c = v[i].z - mean, e = v[i].w - mean;
+        q += (a * a + b * b) + (c * c + e * e);
+      }
+    }
+    const float rstd = rsqrtf(block_sum(q, red) / d + eps);
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const int k = i * blockDim.x + threadIdx.x;
+      if (k < nvec) {
+        const float vals[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const int c = 4 * k + t;
+          Operand<T>::store(ur, d, c, (vals[t] - mean) * rstd * to_f32(gamma[c]) + to_f32(beta[c]));
+        }
+      }
+    }
+    return;
+  }
   float s = 0.f;
   for (int c = threadIdx.x; c < d; c += blockDim.x) s += xr[c];
   const float mean = block_sum(s, red) / d;
   float q = 0.f;
   for (int c = threadIdx.x; c < d; c += blockDim.x) { const float t = xr[c] - mean; q += t * t; }
   const float rstd = rsqrtf(block_sum(q, red) / d + eps);
-  T* ur = u + (size_t)r * d * Operand<T>::PARTS;
   for (int c = threadIdx.x; c < d; c += blockDim.x)
     Operand<T>::store(ur, d, c, (xr[c] - mean) * rstd * to_f32(gamma[c]) + to_f32(beta[c]));
 }
