@@ -197,6 +197,8 @@ def gpu_arm(args, wl, rank, world):
     dec = binding.Decoder(s, weights, B, P, G, plan=(wl.max_layers, wl.min_layers, wl.warmup, G),
                           full_capacity=full_ok, device=str(device))
     stream = dec.stream
+    if args.no_graphs:
+        dec.set_option(binding.SD_OPT_GRAPHS, 0)
     prompts = synth.make_prompts(wl).to(device)
     forced = synth.make_forced_tokens(wl)
     logits0 = torch.empty(B, s.vocab, dtype=torch.float32, device=device)
@@ -345,6 +347,7 @@ def main():
     ap.add_argument("--profile-every", type=int, default=8)
     ap.add_argument("--max-gen-steps", type=int, default=0,
                     help="run only the first N decode steps of each pass (for short profiler captures)")
+    ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA graph replay (profiler runs)")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-rows", type=int, default=1)
