@@ -121,7 +121,7 @@ struct QkvOut {
 
 __host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
 __host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
-__host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/; }
+__host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
 
 template <int NB, int EPI>
 __global__ void __launch_bounds__(192, 1)
@@ -141,6 +141,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * STAGES, accum_bar = full0 + 16 * STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  long long* col_row = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [NB], QKV epilogue only
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * BM, m0 = blockIdx.y * NB;
@@ -225,6 +226,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     pdl_wait();                                   // bias aside, the epilogue reads and writes buffers earlier kernels own
     const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, +32) belong to this warp
     const int n = n0 + quarter * 32 + lane;
+    // QKV epilogue: cache row (b * H * cap + pos) of every token column, worked out once per block;
+    // this thread's feature picks the head and the element inside the row
+    int kv_head = 0, kv_elem = 0;
+    __nv_bfloat16* kv_base = nullptr;
+    if (EPI == EPI_QKV_CACHE) {
+      const int t = threadIdx.x - 64;             // 0..127 over the four epilogue warps
+      if (t < NB) {
+        int b, pos;
+        qo.map.get(m0 + t, b, pos);
+        col_row[t] = (m0 + t < M && pos < qo.cap) ? (long long)b * qo.H * qo.cap + pos : -1;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (n >= qo.d && n < N) {
+        const int cc = n < 2 * qo.d ? n - qo.d : n - 2 * qo.d;
+        kv_head = cc / qo.hd;
+        kv_elem = cc - kv_head * qo.hd;
+        kv_base = n < 2 * qo.d ? qo.Kc : qo.Vc;
+      }
+    }
     if (mbar_wait(accum_bar, 0, abort_flag, status)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const float b = (bias != nullptr && n < N && (EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
@@ -243,15 +263,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               const size_t idx = (size_t)m * ldo + n;
               if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
               else if (EPI == EPI_QKV_CACHE) {
-                if (n < qo.d) {
+                if (kv_base == nullptr) {
                   reinterpret_cast<float*>(out)[idx] = v;
                 } else {
-                  int b, pos;
-                  qo.map.get(m, b, pos);
-                  const int cc = n < 2 * qo.d ? n - qo.d : n - 2 * qo.d;
-                  const int hh = cc / qo.hd, e = cc - hh * qo.hd;
-                  if (pos < qo.cap)
-                    (n < 2 * qo.d ? qo.Kc : qo.Vc)[(((size_t)b * qo.H + hh) * qo.cap + pos) * qo.hd + e] = __float2bfloat16_rn(v);
+                  const long long row = col_row[c + j];
+                  if (row >= 0) kv_base[((size_t)row + (size_t)kv_head * qo.cap) * qo.hd + kv_elem] = __float2bfloat16_rn(v);
                 }
               }
               else if (EPI == EPI_RELU_T)      // the result is the next product's operand: row of 2N bf16, hi | lo

@@ -218,7 +218,7 @@ __device__ __forceinline__ float exp2_safe(float a, float m) {   // 2^(a - m), 0
 }
 
 template <typename T, int HD, int UNROLL>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 7)
 attn_partial_kernel(const float* __restrict__ qkv, int ldq, const T* __restrict__ Kc, const T* __restrict__ Vc,
                     int cap, int H, RowMap map, int chunk, int max_chunks,
                     float* part_acc, float* part_ml, int* __restrict__ counters, T* __restrict__ o) {
