@@ -202,9 +202,11 @@ int sd_launch_count(sd_handle *h, int64_t *launches);
 enum {
   SD_OPT_GRAPHS = 1,       /* 1 (default): replay one CUDA graph per step shape; 0: plain launches */
   SD_OPT_ATTN_CHUNK = 2,   /* keys per split of the decode attention (multiple of 32); 0 = automatic */
-  SD_OPT_GEMM = 3,         /* 0 = automatic; 1 = CUDA-core GEMMs only (bf16 mode as well)          */
+  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (256-row cluster kernel, else 128-row kernel,
+                              else CUDA cores); 1 = CUDA cores only; 2 = 128-row tensor-core kernel   */
   SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
-  SD_OPT_PDL = 5           /* 1 (default): programmatic dependent launch between the step's kernels */
+  SD_OPT_PDL = 5,          /* 1 (default): programmatic dependent launch between the step's kernels */
+  SD_OPT_CLUSTER = 6       /* blocks per cluster that split K in the 256-row GEMM: 0 = automatic, 1..4 */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 

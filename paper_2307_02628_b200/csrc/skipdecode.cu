@@ -14,6 +14,7 @@
 
 #include "kernels.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_wide.cuh"
 
 namespace {
 
@@ -62,6 +63,7 @@ struct sd_handle {
   double k_ms[SD_K_COUNT] = {};
   int64_t k_launches[SD_K_COUNT] = {};
   sd::TcContext tc;
+  sd::WideContext wide;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(arena + off); }
   int* status() const { return at<int>(A.scalars); }
@@ -185,8 +187,10 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, const T* bias, i
   sd_handle* h = Lc.h;
   Lc.begin(cls);
   bool done = false;
-  if (std::is_same<T, bf16>::value && h->opt_gemm != 1)
-    done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status());
+  if (std::is_same<T, bf16>::value && h->opt_gemm != 1) {
+    if (h->opt_gemm == 0) done = sd::wide_gemm(h->wide, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status());
+    if (!done) done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status());
+  }
   if (!done) {
     dim3 grid((N + 63) / 64, (M + 63) / 64);
     const int lda = K * sd::Operand<T>::PARTS;
@@ -211,7 +215,9 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, const
   if (h->opt_gemm == 1) return false;
   const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map};
   Lc.begin(SD_K_GEMM);
-  const bool done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
+  bool done = false;
+  if (h->opt_gemm == 0) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
+  if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
   if (done) Lc.end(); else Lc.cancel();
   return done;
 }
@@ -470,6 +476,7 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
   }
   sd::tc_init(h->tc);
   h->tc.pdl = h->opt_pdl != 0;
+  sd::wide_init(h->wide, h->tc);
   *out = h;
   return SD_OK;
 }
@@ -621,9 +628,13 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != 0 && (value < kMinChunk || value % kMinChunk)) return SD_ERR_ARG;
       h->opt_chunk = value; return SD_OK;
     case SD_OPT_GEMM:
-      if (value < 0 || value > 1) return SD_ERR_ARG;
+      if (value < 0 || value > 2) return SD_ERR_ARG;
       if (value != h->opt_gemm) drop_graphs(h);
       h->opt_gemm = value; return SD_OK;
+    case SD_OPT_CLUSTER:
+      if (value < 0 || value > sd::tcw::MAX_CLUSTER) return SD_ERR_ARG;
+      if (value != h->wide.force_cluster) drop_graphs(h);
+      h->wide.force_cluster = value; return SD_OK;
     case SD_OPT_PDL:
       if ((value != 0) != (h->opt_pdl != 0)) drop_graphs(h);
       h->opt_pdl = value ? 1 : 0; h->tc.pdl = h->opt_pdl != 0; return SD_OK;
