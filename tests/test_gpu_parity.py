@@ -209,15 +209,32 @@ def test_tensor_core_and_cuda_core_gemm_paths_agree(B, P):
     prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
     ref = harness.oracle_run_forced(wl, w, prompts, forced)
     outs = []
-    for mode in (1, 0):
+    for mode in (1, 2, 0):          # CUDA cores, 128-row tcgen05 kernel, 256-row cluster kernel
         dec = harness.make_decoder(wl, w)
         dec.set_option(binding.SD_OPT_GEMM, mode)
         outs.append(harness.gpu_run_forced(dec, wl, prompts, forced))
         dec.close()
         _check(outs[-1], ref, "bf16", f"gemm mode {mode} B{B} P{P}")
-    # same bf16 operands, fp32 accumulation in a different order
     # a different summation order flips some bf16 roundings of the activations: ulp-scale differences
     assert float((outs[0] - outs[1]).abs().max()) < 1e-2
+    assert float((outs[0] - outs[2]).abs().max()) < 1e-2
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 3, 4])
+def test_cluster_split_k_reduce_scatter(cluster):
+    """The 256-row GEMM with K split over 1..4 blocks of a cluster and the accumulator rows
+    exchanged through distributed shared memory (QKV, fc1 and LM head; K = 1024 = 16 k-blocks)."""
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("toy-cluster", 2, 1024, 8, 640, 1111, 64, "bf16")
+    wl = synth.Workload(shape, 37, 6, 5, 2, 1, 0)
+    w = synth.make_weights(shape, seed=10, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced)
+    dec = harness.make_decoder(wl, w)
+    dec.set_option(binding.SD_OPT_CLUSTER, cluster)
+    out = harness.gpu_run_forced(dec, wl, prompts, forced)
+    dec.close()
+    _check(out, ref, "bf16", f"cluster {cluster}")
 
 
 def test_launch_modes_compute_the_same_function():
