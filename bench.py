@@ -199,6 +199,10 @@ def gpu_arm(args, wl, rank, world):
     stream = dec.stream
     if args.no_graphs:
         dec.set_option(binding.SD_OPT_GRAPHS, 0)
+    if args.gemm_mode:
+        dec.set_option(binding.SD_OPT_GEMM, args.gemm_mode)
+    if args.cluster:
+        dec.set_option(binding.SD_OPT_CLUSTER, args.cluster)
     prompts = synth.make_prompts(wl).to(device)
     forced = synth.make_forced_tokens(wl)
     logits0 = torch.empty(B, s.vocab, dtype=torch.float32, device=device)
@@ -318,7 +322,7 @@ def gpu_arm(args, wl, rank, world):
         "step_roofline": {"algorithmic_bytes_per_step": total_bytes, "achieved_gbs": total_bytes / (ms_step / 1e3) / 1e9,
                           "frac_of_measured_hbm": total_bytes / (ms_step / 1e3) / 1e9 / peak,
                           "frac_of_8tbs": total_bytes / (ms_step / 1e3) / 1e9 / 8000.0},
-        "kernel_time_share": {k: v[0] for k, v in kt.items()},
+        "kernel_time_ms": {k: v[0] for k, v in kt.items()}, "kernel_launches_timed": {k: v[1] for k, v in kt.items()},
         "full_layer": full, "prefill_s": t_prefill, "weights_s": t_weights,
         "mean_active_layers": sum(n_active) / len(n_active),
     }
@@ -348,6 +352,8 @@ def main():
     ap.add_argument("--max-gen-steps", type=int, default=0,
                     help="run only the first N decode steps of each pass (for short profiler captures)")
     ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA graph replay (profiler runs)")
+    ap.add_argument("--gemm-mode", type=int, default=0, help="SD_OPT_GEMM (0 automatic, 1 CUDA cores, 2 128-row kernel)")
+    ap.add_argument("--cluster", type=int, default=0, help="SD_OPT_CLUSTER (0 automatic)")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-rows", type=int, default=1)

@@ -212,8 +212,9 @@ int sd_set_option(sd_handle *h, int option, int value);
 
 /* Device time and launch count accumulated per kernel class while SD_OPT_TIMING is
  * on; synchronises the stream.  ms, launches: host. */
-enum { SD_K_EMBED = 0, SD_K_LAYERNORM = 1, SD_K_GEMM = 2, SD_K_KV_APPEND = 3,
-       SD_K_ATTENTION = 4, SD_K_LM_HEAD = 5, SD_K_COUNT = 6 };
+enum { SD_K_EMBED = 0, SD_K_LAYERNORM = 1, SD_K_GEMM_QKV = 2, SD_K_KV_APPEND = 3,
+       SD_K_ATTENTION = 4, SD_K_LM_HEAD = 5, SD_K_GEMM_OUT = 6, SD_K_GEMM_FC1 = 7,
+       SD_K_GEMM_FC2 = 8, SD_K_COUNT = 9 };
 int sd_kernel_time(sd_handle *h, int kernel_class, double *ms, int64_t *launches);
 int sd_kernel_time_reset(sd_handle *h);
 

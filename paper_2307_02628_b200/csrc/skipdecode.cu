@@ -214,7 +214,7 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, const
   sd_handle* h = Lc.h;
   if (h->opt_gemm == 1) return false;
   const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map};
-  Lc.begin(SD_K_GEMM);
+  Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
   if (h->opt_gemm == 0) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
   if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
@@ -266,18 +266,18 @@ void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int
   sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
   if (!launch_qkv_to_cache<T>(Lc, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, d, qkv, Kc, Vc, cap, map)) {
-    launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
+    launch_gemm<T>(Lc, SD_K_GEMM_QKV, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
     Lc.begin(SD_K_KV_APPEND);
     sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::kv_append_kernel<T>, dim3(rows), dim3(256), 0, qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
     Lc.end();
   }
   launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
-  launch_gemm<T>(Lc, SD_K_GEMM, o, (const T*)h->w_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
+  launch_gemm<T>(Lc, SD_K_GEMM_OUT, o, (const T*)h->w_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
   Lc.begin(SD_K_LAYERNORM);
   sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
-  launch_gemm<T>(Lc, SD_K_GEMM, u, (const T*)h->w_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f * sd::Operand<T>::PARTS, sd::EPI_RELU_T);
-  launch_gemm<T>(Lc, SD_K_GEMM, y, (const T*)h->w_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
+  launch_gemm<T>(Lc, SD_K_GEMM_FC1, u, (const T*)h->w_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f * sd::Operand<T>::PARTS, sd::EPI_RELU_T);
+  launch_gemm<T>(Lc, SD_K_GEMM_FC2, y, (const T*)h->w_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
 }
 
 template <typename T>
