@@ -95,7 +95,8 @@ int sd_arena_bytes(const sd_config *cfg, const sd_plan *plan, size_t *out);
 
 /* Creates a handle.  arena: device, 256-byte aligned, arena_bytes >= sd_arena_bytes;
  * it holds the per-layer KV caches [max_batch, n_heads, capacity_l, head_dim] for K
- * and for V, the activation buffers, the split-KV partial results and a status word.
+ * and for V, in bf16 mode a tile-packed copy of every weight matrix (made here, once, on
+ * the stream), the activation buffers, the split-KV partial results and a status word.
  * stream: a cudaStream_t (NULL = the legacy default stream).  The arena's status and
  * counters are cleared on the stream.
  * Errors: SD_ERR_ARG (shape rules above, NULL weights), SD_ERR_CAPACITY (arena too
@@ -202,11 +203,12 @@ int sd_launch_count(sd_handle *h, int64_t *launches);
 enum {
   SD_OPT_GRAPHS = 1,       /* 1 (default): replay one CUDA graph per step shape; 0: plain launches */
   SD_OPT_ATTN_CHUNK = 2,   /* keys per split of the decode attention (multiple of 32); 0 = automatic */
-  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (256-row cluster kernel, else 128-row kernel,
-                              else CUDA cores); 1 = CUDA cores only; 2 = 128-row tensor-core kernel   */
+  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (128-row tensor-core kernel, else CUDA cores);
+                              1 = CUDA cores only; 2 = 128-row kernel; 3 = 256-row cluster kernel      */
   SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
   SD_OPT_PDL = 5,          /* 1 (default): programmatic dependent launch between the step's kernels */
-  SD_OPT_CLUSTER = 6       /* blocks per cluster that split K in the 256-row GEMM: 0 = automatic, 1..4 */
+  SD_OPT_CLUSTER = 6,      /* blocks per cluster that split K in the 256-row GEMM: 0 = automatic, 1..4 */
+  SD_OPT_WEIGHT_TILES = 7  /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 

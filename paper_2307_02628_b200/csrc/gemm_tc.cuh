@@ -117,7 +117,17 @@ struct QkvOut {
   __nv_bfloat16* Vc;
   int d, H, hd, cap;
   RowMap map;
+  int packed_kb;     // every epilogue: 0 = W is row-major [N, K]; else W is tile-packed with K/64 tiles per row tile
 };
+
+// Tile-packed weights: [ceil(N/128)][K/64][128][64] bf16, each 128 x 64 tile a contiguous
+// 16 KB block and the tiles a block streams (fixed row tile, consecutive k-blocks) adjacent, so
+// a block reads one contiguous region of HBM instead of 128-byte pieces 2K bytes apart.
+// The packed matrix is addressed through a tensor map of 64 columns x (tiles * 128) rows.
+__device__ __forceinline__ void load_w_tile(uint32_t dst, const CUtensorMap* map, int packed_kb, int kb, int n_row0, uint32_t bar) {
+  if (packed_kb) tma_load_2d(dst, map, 0, ((n_row0 >> 7) * packed_kb + kb) * BM, bar);
+  else tma_load_2d(dst, map, kb * BK, n_row0, bar);
+}
 
 __host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
 __host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
@@ -175,7 +185,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       for (int i = 0; i < early; ++i) {
         const uint32_t fb = full0 + 8 * i;
         mbar_expect_tx(fb, STAGE_BYTES);
-        tma_load_2d(tiles + i * STAGE_BYTES, &map_w, (kb0 + i) * BK, n0, fb);
+        load_w_tile(tiles + i * STAGE_BYTES, &map_w, qo.packed_kb, kb0 + i, n0, fb);
       }
       pdl_wait();
       int issued = early;
@@ -186,7 +196,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (round > 0) {
           if (!mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
           mbar_expect_tx(fb, STAGE_BYTES);
-          tma_load_2d(a_dst, &map_w, (kb0 + i) * BK, n0, fb);
+          load_w_tile(a_dst, &map_w, qo.packed_kb, kb0 + i, n0, fb);
         }
         tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);                 // hi part: columns [0, K)
         tma_load_2d(a_dst + A_BYTES + B_BYTES, &map_x, K + (kb0 + i) * BK, m0, fb);   // lo part: columns [K, 2K)
@@ -287,6 +297,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   }
 }
 
+// One block per 128 x 64 tile: packed[(tn * KB + kb)][r][c] = W[tn * 128 + r][kb * 64 + c], zero past row N.
+__global__ void pack_tiles_kernel(const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ P, int N, int K) {
+  const int KB = K / BK;
+  const int tn = blockIdx.x / KB, kb = blockIdx.x - tn * KB;
+  uint4* dst = reinterpret_cast<uint4*>(P + (size_t)blockIdx.x * BM * BK);
+  for (int i = threadIdx.x; i < BM * BK / 8; i += blockDim.x) {      // 16-byte pieces: 8 per tile row
+    const int r = i >> 3, c8 = i & 7;
+    const int n = tn * BM + r;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (n < N) v = *reinterpret_cast<const uint4*>(W + (size_t)n * K + kb * BK + c8 * 8);
+    dst[i] = v;
+  }
+}
+
 }  // namespace tc
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -352,6 +376,12 @@ inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int co
   return &c.maps.emplace(key, m).first->second;
 }
 
+// tensor map of a tile-packed weight matrix: 64 columns x (n_tiles * 128) rows, 128-row boxes
+inline const CUtensorMap* tc_map_packed(TcContext& c, const void* ptr, int N, int K) {
+  const int rows = ((N + tc::BM - 1) / tc::BM) * (K / tc::BK) * tc::BM;
+  return tc_map(c, ptr, rows, tc::BK, tc::BM);
+}
+
 template <int NB>
 inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
                       int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status, const tc::QkvOut& qo) {
@@ -370,13 +400,15 @@ inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CU
 
 // Returns true when the product was enqueued on the tensor-core path; false leaves it to the caller.
 inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const __nv_bfloat16* W, const __nv_bfloat16* bias,
-                    int M, int N, int K, void* out, int ldo, int epi, int* status, const tc::QkvOut* qkv_out = nullptr) {
+                    int M, int N, int K, void* out, int ldo, int epi, int* status, const tc::QkvOut* qkv_out = nullptr,
+                    const __nv_bfloat16* Wp = nullptr) {
   if (!c.ready || K % tc::BK || M < 1 || N < 1) return false;   // the hi and lo halves of a row are K apart: whole k-blocks only
   if (epi == EPI_QKV_CACHE && (!qkv_out || qkv_out->d % tc::BM || N != 3 * qkv_out->d)) return false;
-  const tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
+  tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
+  qo.packed_kb = Wp ? K / tc::BK : 0;
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
   const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
-  const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
+  const CUtensorMap* mw = Wp ? tc_map_packed(c, Wp, N, K) : tc_map(c, W, N, K, tc::BM);
   const CUtensorMap* mx = tc_map(c, X, M, 2 * K, nb);
   if (!mw || !mx) return false;
   const int kb_total = (K + tc::BK - 1) / tc::BK;
@@ -396,7 +428,7 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
 }
 template <typename T>
 inline bool tc_gemm(TcContext&, cudaStream_t, const T*, const T*, const T*, int, int, int, void*, int, int, int*,
-                    const tc::QkvOut* = nullptr) {
+                    const tc::QkvOut* = nullptr, const T* = nullptr) {
   return false;                                  // fp32 storage runs on the CUDA-core kernel
 }
 

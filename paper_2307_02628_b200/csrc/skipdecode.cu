@@ -28,6 +28,9 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Arena {            // byte offsets into the caller's arena
   std::vector<size_t> k_off, v_off;
+  std::vector<size_t> wp_qkv, wp_o, wp_fc1, wp_fc2;   // tile-packed copies of the weight matrices (bf16 mode)
+  size_t wp_head;
+  bool packable;
   std::vector<int> cap;
   size_t x, u, qkv, o, y, part_acc, part_ml, counters, row_index, ids, logits, scalars, total;
   int rows_max;
@@ -54,7 +57,8 @@ struct sd_handle {
   int B = 0, P = 0, next_pos = 0;
   int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
-  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = 1;
+  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = 1, opt_tiles = 1;
+  bool packed = false;       // the arena holds tile-packed copies of the weight matrices
   // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
   struct Graph { cudaGraphExec_t exec; int64_t nodes; };
   std::map<std::tuple<int, int, int, int, int, const void*, const void*>, Graph> graphs;
@@ -127,6 +131,19 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
     A.k_off[l] = take(bytes);
     A.v_off[l] = take(bytes);
   }
+  A.packable = c.dtype == SD_DTYPE_BF16 && d % 64 == 0 && c.d_ffn % 64 == 0;
+  A.wp_qkv.assign(L, 0); A.wp_o.assign(L, 0); A.wp_fc1.assign(L, 0); A.wp_fc2.assign(L, 0);
+  A.wp_head = 0;
+  if (A.packable) {
+    auto packed_bytes = [](size_t n, size_t k) { return (n + 127) / 128 * 128 * k * 2; };
+    for (int l = 0; l < L; ++l) {
+      A.wp_qkv[l] = take(packed_bytes(3 * d, d));
+      A.wp_o[l] = take(packed_bytes(d, d));
+      A.wp_fc1[l] = take(packed_bytes(c.d_ffn, d));
+      A.wp_fc2[l] = take(packed_bytes(d, c.d_ffn));
+    }
+    A.wp_head = take(packed_bytes(c.vocab, d));
+  }
   const int chunk_rows = std::max(1, kPrefillTokens / c.max_prompt) * c.max_prompt;
   A.rows_max = std::max(c.max_batch, chunk_rows);
   const size_t R = A.rows_max;
@@ -182,14 +199,15 @@ struct Launcher {
 };
 
 template <typename T>
-void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, const T* bias, int M, int N, int K,
+void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_off, const T* bias, int M, int N, int K,
                  void* out, int ldo, int epi) {
   sd_handle* h = Lc.h;
+  const T* Wp = (h->packed && h->opt_tiles) ? h->at<T>(packed_off) : nullptr;
   Lc.begin(cls);
   bool done = false;
   if (std::is_same<T, bf16>::value && h->opt_gemm != 1) {
-    if (h->opt_gemm == 0) done = sd::wide_gemm(h->wide, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status());
-    if (!done) done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status());
+    if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
+    if (!done) done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
   }
   if (!done) {
     dim3 grid((N + 63) / 64, (M + 63) / 64);
@@ -207,17 +225,18 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, const T* bias, i
 // QKV projection with the K/V rows written straight into the cache by the GEMM epilogue
 // (tensor-core path only).  Returns false when that path does not take the product.
 template <typename T>
-bool launch_qkv_to_cache(Launcher&, const T*, const T*, const T*, int, int, float*, T*, T*, int, sd::RowMap) { return false; }
+bool launch_qkv_to_cache(Launcher&, const T*, const T*, size_t, const T*, int, int, float*, T*, T*, int, sd::RowMap) { return false; }
 template <>
-bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, const bf16* bias, int rows, int d, float* qkv,
+bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_t packed_off, const bf16* bias, int rows, int d, float* qkv,
                                bf16* Kc, bf16* Vc, int cap, sd::RowMap map) {
   sd_handle* h = Lc.h;
   if (h->opt_gemm == 1) return false;
-  const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map};
+  const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map, 0};
+  const bf16* Wp = (h->packed && h->opt_tiles) ? h->at<bf16>(packed_off) : nullptr;
   Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
-  if (h->opt_gemm == 0) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
-  if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo);
+  if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
+  if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (done) Lc.end(); else Lc.cancel();
   return done;
 }
@@ -265,19 +284,19 @@ void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int
   Lc.begin(SD_K_LAYERNORM);
   sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
-  if (!launch_qkv_to_cache<T>(Lc, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, d, qkv, Kc, Vc, cap, map)) {
-    launch_gemm<T>(Lc, SD_K_GEMM_QKV, u, (const T*)h->w_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
+  if (!launch_qkv_to_cache<T>(Lc, u, (const T*)h->w_qkv[l], h->A.wp_qkv[l], (const T*)h->b_qkv[l], rows, d, qkv, Kc, Vc, cap, map)) {
+    launch_gemm<T>(Lc, SD_K_GEMM_QKV, u, (const T*)h->w_qkv[l], h->A.wp_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
     Lc.begin(SD_K_KV_APPEND);
     sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::kv_append_kernel<T>, dim3(rows), dim3(256), 0, qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
     Lc.end();
   }
   launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
-  launch_gemm<T>(Lc, SD_K_GEMM_OUT, o, (const T*)h->w_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
+  launch_gemm<T>(Lc, SD_K_GEMM_OUT, o, (const T*)h->w_o[l], h->A.wp_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
   Lc.begin(SD_K_LAYERNORM);
   sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
-  launch_gemm<T>(Lc, SD_K_GEMM_FC1, u, (const T*)h->w_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f * sd::Operand<T>::PARTS, sd::EPI_RELU_T);
-  launch_gemm<T>(Lc, SD_K_GEMM_FC2, y, (const T*)h->w_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
+  launch_gemm<T>(Lc, SD_K_GEMM_FC1, u, (const T*)h->w_fc1[l], h->A.wp_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f * sd::Operand<T>::PARTS, sd::EPI_RELU_T);
+  launch_gemm<T>(Lc, SD_K_GEMM_FC2, y, (const T*)h->w_fc2[l], h->A.wp_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
 }
 
 template <typename T>
@@ -298,7 +317,7 @@ void enqueue_head(Launcher& Lc, int rows, const int* row_index, float* d_logits)
   sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(c.d_model)), 0, h->at<float>(h->A.x), (const T*)h->lnf_g, (const T*)h->lnf_b,
                                                                         h->at<T>(h->A.u), c.d_model, c.ln_eps, row_index);
   Lc.end();
-  launch_gemm<T>(Lc, SD_K_LM_HEAD, h->at<T>(h->A.u), (const T*)h->lm_head, (const T*)nullptr, rows, c.vocab, c.d_model,
+  launch_gemm<T>(Lc, SD_K_LM_HEAD, h->at<T>(h->A.u), (const T*)h->lm_head, h->A.wp_head, (const T*)nullptr, rows, c.vocab, c.d_model,
                  d_logits, c.vocab, sd::EPI_STORE_F32);
 }
 
@@ -477,6 +496,22 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
   sd::tc_init(h->tc);
   h->tc.pdl = h->opt_pdl != 0;
   sd::wide_init(h->wide, h->tc);
+  if (h->tc.ready && h->A.packable) {            // tile-packed copies of the matrices, made once
+    const int d = cfg->d_model, f = cfg->d_ffn;
+    auto pack = [&](const void* W, size_t off, int n, int k) {
+      const int tiles = (n + 127) / 128 * (k / 64);
+      sd::tc::pack_tiles_kernel<<<tiles, 256, 0, h->stream>>>(static_cast<const bf16*>(W), h->at<bf16>(off), n, k);
+    };
+    for (int l = 0; l < L; ++l) {
+      pack(h->w_qkv[l], h->A.wp_qkv[l], 3 * d, d);
+      pack(h->w_o[l], h->A.wp_o[l], d, d);
+      pack(h->w_fc1[l], h->A.wp_fc1[l], f, d);
+      pack(h->w_fc2[l], h->A.wp_fc2[l], d, f);
+    }
+    pack(h->lm_head, h->A.wp_head, cfg->vocab, d);
+    if (cudaGetLastError() != cudaSuccess) { delete h; return SD_ERR_CUDA; }
+    h->packed = true;
+  }
   *out = h;
   return SD_OK;
 }
@@ -628,13 +663,16 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != 0 && (value < kMinChunk || value % kMinChunk)) return SD_ERR_ARG;
       h->opt_chunk = value; return SD_OK;
     case SD_OPT_GEMM:
-      if (value < 0 || value > 2) return SD_ERR_ARG;
+      if (value < 0 || value > 3) return SD_ERR_ARG;
       if (value != h->opt_gemm) drop_graphs(h);
       h->opt_gemm = value; return SD_OK;
     case SD_OPT_CLUSTER:
       if (value < 0 || value > sd::tcw::MAX_CLUSTER) return SD_ERR_ARG;
       if (value != h->wide.force_cluster) drop_graphs(h);
       h->wide.force_cluster = value; return SD_OK;
+    case SD_OPT_WEIGHT_TILES:
+      if ((value != 0) != (h->opt_tiles != 0)) drop_graphs(h);
+      h->opt_tiles = value ? 1 : 0; return SD_OK;
     case SD_OPT_PDL:
       if ((value != 0) != (h->opt_pdl != 0)) drop_graphs(h);
       h->opt_pdl = value ? 1 : 0; h->tc.pdl = h->opt_pdl != 0; return SD_OK;
