@@ -118,15 +118,23 @@ struct QkvOut {
   int d, H, hd, cap;
   RowMap map;
   int packed_kb;     // every epilogue: 0 = W is row-major [N, K]; else W is tile-packed with K/64 tiles per row tile
+  const __nv_bfloat16* w_packed;
 };
 
-// Tile-packed weights: [ceil(N/128)][K/64][128][64] bf16, each 128 x 64 tile a contiguous
-// 16 KB block and the tiles a block streams (fixed row tile, consecutive k-blocks) adjacent, so
-// a block reads one contiguous region of HBM instead of 128-byte pieces 2K bytes apart.
-// The packed matrix is addressed through a tensor map of 64 columns x (tiles * 128) rows.
-__device__ __forceinline__ void load_w_tile(uint32_t dst, const CUtensorMap* map, int packed_kb, int kb, int n_row0, uint32_t bar) {
-  if (packed_kb) tma_load_2d(dst, map, 0, ((n_row0 >> 7) * packed_kb + kb) * BM, bar);
-  else tma_load_2d(dst, map, kb * BK, n_row0, bar);
+// Tile-packed weights: [ceil(N/128)][K/64] tiles of 128 rows x 64 columns, each tile stored as
+// the 16 KB shared-memory image the MMA wants (128-byte rows with the 128-byte swizzle already
+// applied: 16-byte chunk c of row r sits at chunk c ^ (r & 7)).  A tile is then one contiguous
+// 1-D bulk copy, with no per-row address generation, and the tiles a block streams (fixed row
+// tile, consecutive k-blocks) are adjacent in HBM.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void load_w_tile(uint32_t dst, const CUtensorMap* map, const QkvOut& qo, int kb, int n_row0, uint32_t bar) {
+  if (qo.packed_kb)
+    bulk_load(dst, qo.w_packed + ((size_t)(n_row0 >> 7) * qo.packed_kb + kb) * (BM * BK), BM * BK * 2, bar);
+  else
+    tma_load_2d(dst, map, kb * BK, n_row0, bar);
 }
 
 __host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
@@ -140,7 +148,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                int kb_per_split, int* __restrict__ status, const QkvOut qo) {
   constexpr int STAGES = stages_for(NB);
   constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
-  constexpr int TMEM_COLS = NB < 32 ? 32 : NB;
+  constexpr int TMEM_COLS = 2 * NB;              // W.hi in columns [0, NB), W.lo in [NB, 2 NB): power of two >= 32
   constexpr int CW = NB < 32 ? 16 : 32;          // accumulator columns read per tcgen05.ld
 
   extern __shared__ uint8_t smem_raw[];
@@ -185,7 +193,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       for (int i = 0; i < early; ++i) {
         const uint32_t fb = full0 + 8 * i;
         mbar_expect_tx(fb, STAGE_BYTES);
-        load_w_tile(tiles + i * STAGE_BYTES, &map_w, qo.packed_kb, kb0 + i, n0, fb);
+        load_w_tile(tiles + i * STAGE_BYTES, &map_w, qo, kb0 + i, n0, fb);
       }
       pdl_wait();
       int issued = early;
@@ -196,7 +204,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (round > 0) {
           if (!mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
           mbar_expect_tx(fb, STAGE_BYTES);
-          load_w_tile(a_dst, &map_w, qo.packed_kb, kb0 + i, n0, fb);
+          load_w_tile(a_dst, &map_w, qo, kb0 + i, n0, fb);
         }
         tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);                 // hi part: columns [0, K)
         tma_load_2d(a_dst + A_BYTES + B_BYTES, &map_x, K + (kb0 + i) * BK, m0, fb);   // lo part: columns [K, 2K)
@@ -213,7 +221,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(NB);
+      // The hi tile (NB rows) and the lo tile (NB rows) sit back to back in the stage, so they are
+      // one K-major operand of 2 NB rows: a single MMA of N = 2 NB per k-step puts W.hi and W.lo
+      // side by side in tensor memory (the epilogue adds the halves).  One wide instruction
+      // instead of two narrow ones: at these sizes the MMA pipe is paced per instruction.
+      constexpr uint32_t idesc = instr_desc(2 * NB);
       bool ok = true;
       for (int i = 0; i < nkb && ok; ++i) {
         const int s = i % STAGES, round = i / STAGES;
@@ -221,13 +233,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = tiles + s * STAGE_BYTES;
-        const uint64_t a_desc = smem_desc(a_addr), hi_desc = smem_desc(a_addr + A_BYTES),
-                       lo_desc = smem_desc(a_addr + A_BYTES + B_BYTES);
+        const uint64_t a_desc = smem_desc(a_addr), b_desc = smem_desc(a_addr + A_BYTES);
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k) {   // 32 bytes further along K inside the swizzle row
-          umma(tmem_base, a_desc + 2 * k, hi_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-          umma(tmem_base, a_desc + 2 * k, lo_desc + 2 * k, idesc, 1u);
-        }
+        for (int k = 0; k < BK / UMMA_K; ++k)     // 32 bytes further along K inside the swizzle row
+          umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
         umma_commit(empty0 + 8 * s);              // the stage is free once these MMAs have read it
       }
       if (ok) umma_commit(accum_bar);             // accumulator complete
@@ -260,16 +269,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       const float b = (bias != nullptr && n < N && (EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
 #pragma unroll 1
       for (int c = 0; c < NB; c += CW) {
-        uint32_t r[32];
+        uint32_t r[32], rl[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
-        if (CW == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
+        if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (n < N) {
 #pragma unroll
           for (int j = 0; j < CW; ++j) {
             const int m = m0 + c + j;
             if (m < M) {
-              const float v = __uint_as_float(r[j]) + b;
+              const float v = (__uint_as_float(r[j]) + __uint_as_float(rl[j])) + b;
               const size_t idx = (size_t)m * ldo + n;
               if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
               else if (EPI == EPI_QKV_CACHE) {
@@ -297,7 +306,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   }
 }
 
-// One block per 128 x 64 tile: packed[(tn * KB + kb)][r][c] = W[tn * 128 + r][kb * 64 + c], zero past row N.
+// One block per 128 x 64 tile: tile (tn, kb) holds W[tn * 128 + r][kb * 64 + 8 c .. +8] at 16-byte
+// piece r * 8 + (c ^ (r & 7)); rows past N are zero.
 __global__ void pack_tiles_kernel(const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ P, int N, int K) {
   const int KB = K / BK;
   const int tn = blockIdx.x / KB, kb = blockIdx.x - tn * KB;
@@ -307,7 +317,7 @@ __global__ void pack_tiles_kernel(const __nv_bfloat16* __restrict__ W, __nv_bflo
     const int n = tn * BM + r;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (n < N) v = *reinterpret_cast<const uint4*>(W + (size_t)n * K + kb * BK + c8 * 8);
-    dst[i] = v;
+    dst[r * 8 + (c8 ^ (r & 7))] = v;
   }
 }
 
@@ -376,12 +386,6 @@ inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int co
   return &c.maps.emplace(key, m).first->second;
 }
 
-// tensor map of a tile-packed weight matrix: 64 columns x (n_tiles * 128) rows, 128-row boxes
-inline const CUtensorMap* tc_map_packed(TcContext& c, const void* ptr, int N, int K) {
-  const int rows = ((N + tc::BM - 1) / tc::BM) * (K / tc::BK) * tc::BM;
-  return tc_map(c, ptr, rows, tc::BK, tc::BM);
-}
-
 template <int NB>
 inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
                       int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status, const tc::QkvOut& qo) {
@@ -406,9 +410,10 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   if (epi == EPI_QKV_CACHE && (!qkv_out || qkv_out->d % tc::BM || N != 3 * qkv_out->d)) return false;
   tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
   qo.packed_kb = Wp ? K / tc::BK : 0;
+  qo.w_packed = Wp;
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
   const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
-  const CUtensorMap* mw = Wp ? tc_map_packed(c, Wp, N, K) : tc_map(c, W, N, K, tc::BM);
+  const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);      // unused by the kernel when the packed copy is read
   const CUtensorMap* mx = tc_map(c, X, M, 2 * K, nb);
   if (!mw || !mx) return false;
   const int kb_total = (K + tc::BK - 1) / tc::BK;

@@ -103,8 +103,8 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
       for (int i = 0; i < early; ++i) {
         const uint32_t fb = full0 + 8 * i, dst = tiles + i * STAGE_BYTES;
         mbar_expect_tx(fb, STAGE_BYTES);
-        load_w_tile(dst, &map_w, qo.packed_kb, kb0 + i, n0, fb);
-        load_w_tile(dst + A_HALF, &map_w, qo.packed_kb, kb0 + i, n0 + 128, fb);
+        load_w_tile(dst, &map_w, qo, kb0 + i, n0, fb);
+        load_w_tile(dst + A_HALF, &map_w, qo, kb0 + i, n0 + 128, fb);
       }
       pdl_wait();
       int issued = early;
@@ -114,8 +114,8 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         if (round > 0) {
           if (!mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
           mbar_expect_tx(fb, STAGE_BYTES);
-          load_w_tile(dst, &map_w, qo.packed_kb, kb0 + i, n0, fb);
-          load_w_tile(dst + A_HALF, &map_w, qo.packed_kb, kb0 + i, n0 + 128, fb);
+          load_w_tile(dst, &map_w, qo, kb0 + i, n0, fb);
+          load_w_tile(dst + A_HALF, &map_w, qo, kb0 + i, n0 + 128, fb);
         }
         tma_load_2d(dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);
         tma_load_2d(dst + A_BYTES + B_BYTES, &map_x, K + (kb0 + i) * BK, m0, fb);
@@ -332,8 +332,9 @@ inline bool wide_gemm(WideContext& w, TcContext& c, cudaStream_t st, const __nv_
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
   tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
   qo.packed_kb = Wp ? K / tc::BK : 0;
+  qo.w_packed = Wp;
   const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
-  const CUtensorMap* mw = Wp ? tc_map_packed(c, Wp, N, K) : tc_map(c, W, N, K, tc::BM);
+  const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
   const CUtensorMap* mx = tc_map(c, X, M, 2 * K, nb);
   if (!mw || !mx) return false;
   const int kb_total = K / tc::BK;

@@ -135,7 +135,7 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   A.wp_qkv.assign(L, 0); A.wp_o.assign(L, 0); A.wp_fc1.assign(L, 0); A.wp_fc2.assign(L, 0);
   A.wp_head = 0;
   if (A.packable) {
-    auto packed_bytes = [](size_t n, size_t k) { return (n + 127) / 128 * 128 * k * 2; };
+    auto packed_bytes = [](size_t n, size_t k) { return (n + 255) / 256 * 256 * k * 2; };   // whole 256-row pairs of tiles
     for (int l = 0; l < L; ++l) {
       A.wp_qkv[l] = take(packed_bytes(3 * d, d));
       A.wp_o[l] = take(packed_bytes(d, d));
@@ -231,7 +231,7 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
                                bf16* Kc, bf16* Vc, int cap, sd::RowMap map) {
   sd_handle* h = Lc.h;
   if (h->opt_gemm == 1) return false;
-  const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map, 0};
+  const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map, 0, nullptr};
   const bf16* Wp = (h->packed && h->opt_tiles) ? h->at<bf16>(packed_off) : nullptr;
   Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
@@ -499,7 +499,7 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
   if (h->tc.ready && h->A.packable) {            // tile-packed copies of the matrices, made once
     const int d = cfg->d_model, f = cfg->d_ffn;
     auto pack = [&](const void* W, size_t off, int n, int k) {
-      const int tiles = (n + 127) / 128 * (k / 64);
+      const int tiles = (n + 255) / 256 * 2 * (k / 64);
       sd::tc::pack_tiles_kernel<<<tiles, 256, 0, h->stream>>>(static_cast<const bf16*>(W), h->at<bf16>(off), n, k);
     };
     for (int l = 0; l < L; ++l) {
