@@ -53,7 +53,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                  int kb_per_split, int* __restrict__ status, const QkvOut qo) {
   constexpr int STAGES = stages_for(NB);
   constexpr int A_BYTES = ROWS * BK * 2, A_HALF = A_BYTES / 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
-  constexpr int TMEM_COLS = 2 * NB < 32 ? 32 : 2 * NB;
+  constexpr int TMEM_COLS = 4 * NB;             // per accumulator: W.hi in [0, NB), W.lo in [NB, 2 NB)
   constexpr int CW = NB < 32 ? 16 : 32;
 
   extern __shared__ uint8_t smem_raw[];
@@ -131,7 +131,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     }
   } else if (warp == 1) {
     if (lane == 0 && nkb > 0) {
-      constexpr uint32_t idesc = instr_desc(NB);
+      constexpr uint32_t idesc = instr_desc(2 * NB);   // hi and lo tiles back to back = one operand of 2 NB rows
       bool ok = true;
       for (int i = 0; i < nkb && ok; ++i) {
         const int s = i % STAGES, round = i / STAGES;
@@ -139,15 +139,12 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = tiles + s * STAGE_BYTES;
-        const uint64_t a0 = smem_desc(a_addr), a1 = smem_desc(a_addr + A_HALF), hi = smem_desc(a_addr + A_BYTES),
-                       lo = smem_desc(a_addr + A_BYTES + B_BYTES);
+        const uint64_t a0 = smem_desc(a_addr), a1 = smem_desc(a_addr + A_HALF), bd = smem_desc(a_addr + A_BYTES);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k) {
           const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
-          umma(tmem_base, a0 + 2 * k, hi + 2 * k, idesc, acc);
-          umma(tmem_base, a0 + 2 * k, lo + 2 * k, idesc, 1u);
-          umma(tmem_base + NB, a1 + 2 * k, hi + 2 * k, idesc, acc);
-          umma(tmem_base + NB, a1 + 2 * k, lo + 2 * k, idesc, 1u);
+          umma(tmem_base, a0 + 2 * k, bd + 2 * k, idesc, acc);
+          umma(tmem_base + 2 * NB, a1 + 2 * k, bd + 2 * k, idesc, acc);
         }
         umma_commit(empty0 + 8 * s);
       }
@@ -184,12 +181,13 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const uint32_t dst0 = map_to_cta(tiles, (uint32_t)owner) + (uint32_t)(((slot * (S - 1) + src) * NB) * 32 + lane) * 4u;
 #pragma unroll 1
         for (int c = 0; c < NB; c += CW) {
-          uint32_t r[32];
-          const uint32_t taddr = tmem_base + lane_base + (uint32_t)(a * NB + c);
-          if (CW == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
+          uint32_t r[32], rl[32];
+          const uint32_t taddr = tmem_base + lane_base + (uint32_t)(a * 2 * NB + c);
+          if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-          for (int j = 0; j < CW; ++j) st_cluster_f32(dst0 + (uint32_t)((c + j) * 32) * 4u, __uint_as_float(r[j]));
+          for (int j = 0; j < CW; ++j)
+            st_cluster_f32(dst0 + (uint32_t)((c + j) * 32) * 4u, __uint_as_float(r[j]) + __uint_as_float(rl[j]));
         }
       }
     }
@@ -216,16 +214,16 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
       }
 #pragma unroll 1
       for (int c = 0; c < NB; c += CW) {
-        uint32_t r[32];
-        const uint32_t taddr = tmem_base + lane_base + (uint32_t)(a * NB + c);
-        if (CW == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
+        uint32_t r[32], rl[32];
+        const uint32_t taddr = tmem_base + lane_base + (uint32_t)(a * 2 * NB + c);
+        if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (n < N) {
 #pragma unroll
           for (int j = 0; j < CW; ++j) {
             const int m = m0 + c + j;
             if (m < M) {
-              float v = __uint_as_float(r[j]) + b;
+              float v = (__uint_as_float(r[j]) + __uint_as_float(rl[j])) + b;
               if (exchange) {
                 for (int s = 0; s < S - 1; ++s) v += recv[((slot * (S - 1) + s) * NB + (c + j)) * 32 + lane];
               }
