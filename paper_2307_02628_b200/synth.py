@@ -69,6 +69,9 @@ CONFIGS = {
     "c3": Workload(OPT_1B3, 32, 512, 256, 24, 8),
     "c4": Workload(OPT_6B7, 64, 1024, 512, 32, 8),
     "c5": Workload(OPT_6B7, 256, 256, 1024, 32, 4),
+    # profiler case: config 4's kernels (same d, heads, batch, prompt, hence the same attention and GEMM
+    # launches) on a 2-layer model, so that a counter capture holds a few GB instead of 60
+    "c4-2layer": Workload(ModelShape("opt-6.7b-2layer", 2, 4096, 32, 16384, 50272, 2048, "bf16"), 64, 1024, 16, 2, 2),
 }
 
 
