@@ -203,6 +203,8 @@ def gpu_arm(args, wl, rank, world):
         dec.set_option(binding.SD_OPT_GEMM, args.gemm_mode)
     if args.cluster:
         dec.set_option(binding.SD_OPT_CLUSTER, args.cluster)
+    if args.attn_chunk:
+        dec.set_option(binding.SD_OPT_ATTN_CHUNK, args.attn_chunk)
     if args.row_major_weights:
         dec.set_option(binding.SD_OPT_WEIGHT_TILES, 0)
     prompts = synth.make_prompts(wl).to(device)
@@ -357,6 +359,7 @@ def main():
     ap.add_argument("--gemm-mode", type=int, default=0, help="SD_OPT_GEMM (0 automatic, 1 CUDA cores, 2 128-row kernel)")
     ap.add_argument("--cluster", type=int, default=0, help="SD_OPT_CLUSTER (0 automatic)")
     ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
+    ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-rows", type=int, default=1)
