@@ -66,6 +66,24 @@ def step_bytes(wl: synth.Workload, n_active) -> float:
     return total
 
 
+# --------------------------------------------------------------------------- ncu traffic of the dominant kernel
+
+# DRAM bytes (read + write) per algorithmic byte of attn_partial_kernel, from the ncu --set full
+# capture summarised in profiles/ncu_full_attn_partial_c4_shape.md (1.08695 GB moved for 1.07583 GB
+# of K and V at T = 1026; the traffic is proportional to T).  Valid only for the kernel source it was
+# taken on: the hash below is checked and `traffic` is null once the kernel text has changed.
+ATTN_TRAFFIC_RATIO = 1.0104
+ATTN_KERNEL_SHA256 = "1869cf8f40bc46c57d62cbbb198d42064b05ac355f561f429b98728d11566cd2"
+
+
+def attention_kernel_hash() -> str:
+    import hashlib
+    src = open(os.path.join(ROOT, "paper_2307_02628_b200", "csrc", "kernels.cuh")).read()
+    i = src.index("template <typename T, int HD, int UNROLL>")
+    j = src.index("// Host side: launch with the programmatic")
+    return hashlib.sha256(src[i:j].encode()).hexdigest()
+
+
 # --------------------------------------------------------------------------- clocks
 
 class ClockSampler:
@@ -321,7 +339,9 @@ def gpu_arm(args, wl, rank, world):
                 "d2h_bytes_per_step": G_run * B * s.vocab * 4},
         "roofline": {"kernel": "attn_partial_kernel (split-KV decode attention)", "bound": "hbm", "achieved": achieved,
                      "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
-                     "traffic": None, "launches_timed": int(attn_n),
+                     "traffic": (ATTN_TRAFFIC_RATIO * attn_bytes / attn_n
+                                 if attn_n and attention_kernel_hash() == ATTN_KERNEL_SHA256 and s.dtype == "bf16" else None),
+                     "launches_timed": int(attn_n),
                      "algorithmic_bytes_per_launch": attn_bytes / attn_n if attn_n else None},
         "step_roofline": {"algorithmic_bytes_per_step": total_bytes, "achieved_gbs": total_bytes / (ms_step / 1e3) / 1e9,
                           "frac_of_measured_hbm": total_bytes / (ms_step / 1e3) / 1e9 / peak,
