@@ -321,15 +321,25 @@ void enqueue_head(Launcher& Lc, int rows, const int* row_index, float* d_logits)
                  d_logits, c.vocab, sd::EPI_STORE_F32);
 }
 
-// keys per split for a decode step with `rows` x H query-heads and T keys each
+// Keys per split for a decode step with `rows` x H query-heads and T keys each: the candidate
+// that minimises (waves of blocks) x (keys a block walks + a fixed cost in key units).  Many
+// (row, head) pairs -> one block walks the whole row (no partials at all); few -> short
+// splits so that every SM has blocks.
 int pick_chunk(const sd_handle* h, int rows, int T) {
   if (h->opt_chunk > 0) return h->opt_chunk;
   const long rh = (long)rows * h->cfg.n_heads;
-  const long want = 8L * 148;                       // blocks in flight to cover the SMs
-  for (int chunk : {512, 256, 128, 64}) {
-    if (rh * ((T + chunk - 1) / chunk) >= want) return chunk;
+  const long slots = 7L * h->tc.sm_count;           // blocks resident at once (7 per SM by registers)
+  const int whole = (h->cfg.max_prompt + h->cfg.max_gen + kMinChunk - 1) / kMinChunk * kMinChunk;
+  int best = whole;
+  double best_cost = 1e30;
+  for (int chunk : {whole, 1024, 768, 512, 256, 128, 64, kMinChunk}) {
+    if (chunk > whole) continue;
+    const long n_chunks = (T + chunk - 1) / chunk;
+    const long waves = (rh * n_chunks + slots - 1) / slots;
+    const double cost = (double)waves * (std::min(chunk, T) + 48);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = chunk; }
   }
-  return kMinChunk;
+  return best;
 }
 
 template <typename T>
