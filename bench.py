@@ -221,6 +221,8 @@ def gpu_arm(args, wl, rank, world):
         dec.set_option(binding.SD_OPT_GEMM, args.gemm_mode)
     if args.cluster:
         dec.set_option(binding.SD_OPT_CLUSTER, args.cluster)
+    if args.no_pdl:
+        dec.set_option(binding.SD_OPT_PDL, 0)
     if args.attn_chunk:
         dec.set_option(binding.SD_OPT_ATTN_CHUNK, args.attn_chunk)
     if args.row_major_weights:
@@ -238,12 +240,13 @@ def gpu_arm(args, wl, rank, world):
 
     G_run = G if args.max_gen_steps <= 0 else min(G, args.max_gen_steps)   # < G only for profiler runs
 
-    def one_pass():
-        dec.rewind()
-        dec.greedy(logits0, ids)
-        for g in range(G_run):
-            dec.decode_step(ids, P + g, logits)
-            dec.greedy(logits, ids)
+    def one_pass(nsteps=None, d=None):
+        d = d or dec
+        d.rewind()
+        d.greedy(logits0, ids)
+        for g in range(G_run if nsteps is None else nsteps):
+            d.decode_step(ids, P + g, logits)
+            d.greedy(logits, ids)
 
     def timed(fn, reps):
         barrier()
@@ -325,6 +328,35 @@ def gpu_arm(args, wl, rank, world):
             full = {"ms_per_step": ms_full, "tokens_per_s": world * B * G_run / (ms_full / 1e3),
                     "speedup_skip_over_full": ms_full / ms_step,
                     "byte_model_bound": step_bytes(wl, [s.n_layers] * G_run) / step_bytes(wl, n_active[:G_run])}
+        elif not args.no_full_layer and G_run == G:
+            # The all-layers cache for the whole generation does not fit beside the weights (config 5:
+            # 172 GB): compare over the longest prefix of positions whose full cache does fit, skip and
+            # full-layer both timed on exactly those positions.
+            free_now, _ = torch.cuda.mem_get_info(device)
+            mine = dec.arena_bytes
+            Gp = 0
+            for cand in range(G - G % 64, 0, -64):
+                need = binding.arena_bytes(binding.make_config(s, B, P, cand), binding.SdPlan(s.n_layers, s.n_layers, 0, cand, 1))
+                if need + (6 << 30) < free_now + mine + wbytes:     # this decoder (arena, device weights) is released first
+                    Gp = cand
+                    break
+            if Gp:
+                one_pass(Gp)
+                ms_skip_p = timed(lambda: one_pass(Gp), max(1, min(2, args.steps)))
+                dec.close()
+                torch.cuda.empty_cache()
+                dec2 = binding.Decoder(s, weights, B, P, Gp, plan=(s.n_layers, s.n_layers, 0, Gp), full_capacity=True,
+                                       device=str(device), stream=stream)
+                dec2.schedule(s.n_layers, s.n_layers, 0, Gp)
+                dec2.prefill(prompts, logits0)
+                one_pass(Gp, dec2)
+                ms_full_p = timed(lambda: one_pass(Gp, dec2), max(1, min(2, args.steps)))
+                assert dec2.status() == 0
+                dec2.close()
+                full = {"prefix_steps": Gp, "ms_full": ms_full_p, "ms_skip_same_steps": ms_skip_p,
+                        "speedup_skip_over_full": ms_full_p / ms_skip_p,
+                        "byte_model_bound": step_bytes(wl, [s.n_layers] * Gp) / step_bytes(wl, n_active[:Gp]),
+                        "note": f"all-layers cache for all {G} steps does not fit; both timed on the first {Gp} positions"}
 
     peak, peak_kind = measured_peaks()
     value = world * B * G_run / (ms_step / 1e3)
@@ -380,6 +412,7 @@ def main():
     ap.add_argument("--cluster", type=int, default=0, help="SD_OPT_CLUSTER (0 automatic)")
     ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
+    ap.add_argument("--no-pdl", action="store_true", help="SD_OPT_PDL = 0")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-rows", type=int, default=1)
