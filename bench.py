@@ -221,8 +221,8 @@ def gpu_arm(args, wl, rank, world):
         dec.set_option(binding.SD_OPT_GEMM, args.gemm_mode)
     if args.cluster:
         dec.set_option(binding.SD_OPT_CLUSTER, args.cluster)
-    if args.no_pdl:
-        dec.set_option(binding.SD_OPT_PDL, 0)
+    if args.pdl is not None:
+        dec.set_option(binding.SD_OPT_PDL, args.pdl)
     if args.attn_chunk:
         dec.set_option(binding.SD_OPT_ATTN_CHUNK, args.attn_chunk)
     if args.row_major_weights:
@@ -412,7 +412,7 @@ def main():
     ap.add_argument("--cluster", type=int, default=0, help="SD_OPT_CLUSTER (0 automatic)")
     ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
-    ap.add_argument("--no-pdl", action="store_true", help="SD_OPT_PDL = 0")
+    ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-rows", type=int, default=1)

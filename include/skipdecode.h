@@ -206,11 +206,17 @@ enum {
   SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (128-row tensor-core kernel, else CUDA cores);
                               1 = CUDA cores only; 2 = 128-row kernel; 3 = 256-row cluster kernel      */
   SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
-  SD_OPT_PDL = 5,          /* 1 (default): programmatic dependent launch between the step's kernels */
+  SD_OPT_PDL = 5,          /* programmatic dependent launch: mask of kernel classes (1 << SD_K_*) whose
+                              kernels may begin before their predecessor ends; 0 = none             */
   SD_OPT_CLUSTER = 6,      /* blocks per cluster that split K in the 256-row GEMM: 0 = automatic, 1..4 */
   SD_OPT_WEIGHT_TILES = 7  /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
 };
 int sd_set_option(sd_handle *h, int option, int value);
+#define SD_PDL_ALL 0x1ff
+/* Default: the five GEMM classes.  A GEMM that starts early sets up its barriers and tensor
+ * memory and streams its first weight tiles while its predecessor drains (measured +1.5 % at the
+ * OPT-6.7B shape); starting the attention kernel or the LayerNorms early costs 2-5 %. */
+#define SD_PDL_DEFAULT ((1 << 2) | (1 << 5) | (1 << 6) | (1 << 7) | (1 << 8))
 
 /* Device time and launch count accumulated per kernel class while SD_OPT_TIMING is
  * on; synchronises the stream.  ms, launches: host. */

@@ -57,7 +57,7 @@ struct sd_handle {
   int B = 0, P = 0, next_pos = 0;
   int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
-  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = 1, opt_tiles = 1;
+  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = SD_PDL_DEFAULT, opt_tiles = 1;
   bool packed = false;       // the arena holds tile-packed copies of the weight matrices
   // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
   struct Graph { cudaGraphExec_t exec; int64_t nodes; };
@@ -198,11 +198,16 @@ struct Launcher {
   }
 };
 
+// SD_OPT_PDL is a mask over kernel classes (bit = 1 << class): a kernel of a class whose bit is
+// set is launched with the programmatic attribute, i.e. may begin before its predecessor ends.
+bool pdl_for(const sd_handle* h, int cls) { return (h->opt_pdl >> cls) & 1; }
+
 template <typename T>
 void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_off, const T* bias, int M, int N, int K,
                  void* out, int ldo, int epi) {
   sd_handle* h = Lc.h;
   const T* Wp = (h->packed && h->opt_tiles) ? h->at<T>(packed_off) : nullptr;
+  h->tc.pdl = pdl_for(h, cls);
   Lc.begin(cls);
   bool done = false;
   if (std::is_same<T, bf16>::value && h->opt_gemm != 1) {
@@ -213,11 +218,11 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_of
     dim3 grid((N + 63) / 64, (M + 63) / 64);
     const int lda = K * sd::Operand<T>::PARTS;
     if (epi == sd::EPI_STORE_F32)
-      sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::gemm_simt_kernel<T, sd::EPI_STORE_F32>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
+      sd::launch_kernel(pdl_for(h, cls), h->stream, sd::gemm_simt_kernel<T, sd::EPI_STORE_F32>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
     else if (epi == sd::EPI_RELU_T)
-      sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::gemm_simt_kernel<T, sd::EPI_RELU_T>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
+      sd::launch_kernel(pdl_for(h, cls), h->stream, sd::gemm_simt_kernel<T, sd::EPI_RELU_T>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
     else
-      sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
+      sd::launch_kernel(pdl_for(h, cls), h->stream, sd::gemm_simt_kernel<T, sd::EPI_RESIDUAL_F32>, dim3(grid), dim3(256), 0, A, lda, W, K, bias, M, N, K, out, ldo);
   }
   Lc.end();
 }
@@ -233,6 +238,7 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
   if (h->opt_gemm == 1) return false;
   const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map, 0, nullptr};
   const bf16* Wp = (h->packed && h->opt_tiles) ? h->at<bf16>(packed_off) : nullptr;
+  h->tc.pdl = pdl_for(h, SD_K_GEMM_QKV);
   Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
   if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
@@ -248,7 +254,7 @@ void launch_attention_hd(Launcher& Lc, const T* Kc, const T* Vc, int cap, int ro
   const int H = h->cfg.n_heads;
   Lc.begin(SD_K_ATTENTION);
   dim3 grid(rows * H, n_chunks);
-  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::attn_partial_kernel<T, HD, 4>, dim3(grid), dim3(128), 0, h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml,
+  sd::launch_kernel(pdl_for(h, SD_K_ATTENTION), h->stream, sd::attn_partial_kernel<T, HD, 4>, dim3(grid), dim3(128), 0, h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml,
       h->at<int>(h->A.counters), h->at<T>(h->A.o));
   Lc.end();
 }
@@ -282,18 +288,18 @@ void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int
   const int cap = h->A.cap[l];
 
   Lc.begin(SD_K_LAYERNORM);
-  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
+  sd::launch_kernel(pdl_for(h, SD_K_LAYERNORM), h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln1_g[l], (const T*)h->ln1_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
   if (!launch_qkv_to_cache<T>(Lc, u, (const T*)h->w_qkv[l], h->A.wp_qkv[l], (const T*)h->b_qkv[l], rows, d, qkv, Kc, Vc, cap, map)) {
     launch_gemm<T>(Lc, SD_K_GEMM_QKV, u, (const T*)h->w_qkv[l], h->A.wp_qkv[l], (const T*)h->b_qkv[l], rows, 3 * d, d, qkv, 3 * d, sd::EPI_STORE_F32);
     Lc.begin(SD_K_KV_APPEND);
-    sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::kv_append_kernel<T>, dim3(rows), dim3(256), 0, qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
+    sd::launch_kernel(pdl_for(h, SD_K_KV_APPEND), h->stream, sd::kv_append_kernel<T>, dim3(rows), dim3(256), 0, qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
     Lc.end();
   }
   launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
   launch_gemm<T>(Lc, SD_K_GEMM_OUT, o, (const T*)h->w_o[l], h->A.wp_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
   Lc.begin(SD_K_LAYERNORM);
-  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
+  sd::launch_kernel(pdl_for(h, SD_K_LAYERNORM), h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
   Lc.end();
   launch_gemm<T>(Lc, SD_K_GEMM_FC1, u, (const T*)h->w_fc1[l], h->A.wp_fc1[l], (const T*)h->b_fc1[l], rows, f, d, y, f * sd::Operand<T>::PARTS, sd::EPI_RELU_T);
   launch_gemm<T>(Lc, SD_K_GEMM_FC2, y, (const T*)h->w_fc2[l], h->A.wp_fc2[l], (const T*)h->b_fc2[l], rows, d, f, x, d, sd::EPI_RESIDUAL_F32);
@@ -303,7 +309,7 @@ template <typename T>
 void enqueue_embed(Launcher& Lc, const int32_t* ids, int rows, sd::RowMap map) {
   sd_handle* h = Lc.h;
   Lc.begin(SD_K_EMBED);
-  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::embed_pos_kernel<T>, dim3(rows), dim3(256), 0, ids, (const T*)h->tok_emb, (const T*)h->pos_emb, h->at<float>(h->A.x),
+  sd::launch_kernel(pdl_for(h, SD_K_EMBED), h->stream, sd::embed_pos_kernel<T>, dim3(rows), dim3(256), 0, ids, (const T*)h->tok_emb, (const T*)h->pos_emb, h->at<float>(h->A.x),
                                                       h->cfg.d_model, h->cfg.vocab, h->cfg.max_pos, map, h->status());
   Lc.end();
 }
@@ -314,7 +320,7 @@ void enqueue_head(Launcher& Lc, int rows, const int* row_index, float* d_logits)
   sd_handle* h = Lc.h;
   const sd_config& c = h->cfg;
   Lc.begin(SD_K_LAYERNORM);
-  sd::launch_kernel(h->opt_pdl != 0, h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(c.d_model)), 0, h->at<float>(h->A.x), (const T*)h->lnf_g, (const T*)h->lnf_b,
+  sd::launch_kernel(pdl_for(h, SD_K_LAYERNORM), h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(c.d_model)), 0, h->at<float>(h->A.x), (const T*)h->lnf_g, (const T*)h->lnf_b,
                                                                         h->at<T>(h->A.u), c.d_model, c.ln_eps, row_index);
   Lc.end();
   launch_gemm<T>(Lc, SD_K_LM_HEAD, h->at<T>(h->A.u), (const T*)h->lm_head, h->A.wp_head, (const T*)nullptr, rows, c.vocab, c.d_model,
@@ -504,7 +510,6 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
     cudaGetLastError(); delete h; return SD_ERR_CUDA;
   }
   sd::tc_init(h->tc);
-  h->tc.pdl = h->opt_pdl != 0;
   sd::wide_init(h->wide, h->tc);
   if (h->tc.ready && h->A.packable) {            // tile-packed copies of the matrices, made once
     const int d = cfg->d_model, f = cfg->d_ffn;
@@ -684,8 +689,9 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if ((value != 0) != (h->opt_tiles != 0)) drop_graphs(h);
       h->opt_tiles = value ? 1 : 0; return SD_OK;
     case SD_OPT_PDL:
-      if ((value != 0) != (h->opt_pdl != 0)) drop_graphs(h);
-      h->opt_pdl = value ? 1 : 0; h->tc.pdl = h->opt_pdl != 0; return SD_OK;
+      if (value < 0 || value >= (1 << SD_K_COUNT)) return SD_ERR_ARG;
+      if (value != h->opt_pdl) drop_graphs(h);
+      h->opt_pdl = value; return SD_OK;
     case SD_OPT_TIMING:
       if (h->opt_timing && !value) collect_timing(h);
       h->opt_timing = value ? 1 : 0; return SD_OK;

@@ -247,7 +247,7 @@ def test_launch_modes_compute_the_same_function():
         prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
         ref = harness.oracle_run_forced(wl, w, prompts, forced)
         for graphs in (1, 0):
-            for pdl in (1, 0):
+            for pdl in (0x1ff, 0):
                 dec = harness.make_decoder(wl, w)
                 dec.set_option(binding.SD_OPT_GRAPHS, graphs)
                 dec.set_option(binding.SD_OPT_PDL, pdl)
