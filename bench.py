@@ -337,7 +337,7 @@ def gpu_arm(args, wl, rank, world):
             Gp = 0
             for cand in range(G - G % 64, 0, -64):
                 need = binding.arena_bytes(binding.make_config(s, B, P, cand), binding.SdPlan(s.n_layers, s.n_layers, 0, cand, 1))
-                if need + (6 << 30) < free_now + mine + wbytes:     # this decoder (arena, device weights) is released first
+                if need + (4 << 30) < free_now + mine:     # this decoder is released first; the next one uploads the weights again
                     Gp = cand
                     break
             if Gp:
