@@ -126,6 +126,21 @@ int sd_schedule(sd_handle *h, int max_layers, int min_layers, int warmup, int ge
 int sd_schedule_compute(int n_layers, int max_layers, int min_layers, int warmup, int gen_len,
                         int32_t *n_active, int32_t *top_begin);
 
+/* Power-law decay, the other budget function Section 2.3 names (host only):
+ *     n_active[g] = round_half_up(min_layers + (max_layers - min_layers) * (1 - t)^alpha),  t = g / (gen_len - 1)
+ * with an integer exponent 1 <= alpha <= 8, computed in integers; alpha = 1 is the linear schedule and
+ * alpha > 1 never exceeds it, so a plan sized for the linear schedule holds every alpha.
+ * Errors: SD_ERR_ARG. */
+int sd_schedule_power_compute(int n_layers, int max_layers, int min_layers, int warmup, int gen_len, int alpha,
+                              int32_t *n_active, int32_t *top_begin);
+
+/* Installs a caller-supplied budget table ("this function can adopt multiple forms", Section 2.3):
+ * n_active: host, gen_len int32, non-increasing (Section 2.2), warmup < n_active[g] <= n_layers.
+ * The layers that run at g are [0, warmup) and [n_layers - (n_active[g] - warmup), n_layers).
+ * top_begin: host, gen_len int32, may be NULL.  Same effects and capacity rule as sd_schedule.
+ * Errors: SD_ERR_ARG (also for a table that grows), SD_ERR_CAPACITY. */
+int sd_schedule_custom(sd_handle *h, const int32_t *n_active, int warmup, int gen_len, int32_t *top_begin);
+
 /* Cache positions the plan reserves per layer (host only): capacity[n_layers]. */
 int sd_layer_capacity(const sd_config *cfg, const sd_plan *plan, int32_t *capacity);
 

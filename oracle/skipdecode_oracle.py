@@ -87,6 +87,21 @@ def schedule(max_layers: int, min_layers: int, warmup: int, gen_len: int, n_laye
     return n_active, top_begin
 
 
+def schedule_power(max_layers: int, min_layers: int, warmup: int, gen_len: int, n_layers: int, alpha: int):
+    """Power-law decay, which Section 2.3 names as another possible budget function:
+    min + (max - min) * (1 - t)^alpha with t = g / (gen_len - 1) (reading: integer exponent,
+    same closed interval and rounding as the linear schedule; alpha = 1 is that schedule)."""
+    if not (0 <= warmup < min_layers <= max_layers <= n_layers and gen_len >= 1 and alpha >= 1):
+        raise ValueError("bad schedule arguments")
+    n_active, top_begin = [], []
+    for g in range(gen_len):
+        t = Fraction(0) if gen_len == 1 else Fraction(g, gen_len - 1)
+        n = math.floor(min_layers + (max_layers - min_layers) * (1 - t) ** alpha + Fraction(1, 2))
+        n_active.append(n)
+        top_begin.append(n_layers - (n - warmup))
+    return n_active, top_begin
+
+
 def active_layers(n_layers: int, n: int, warmup: int):
     """Indices of the layers that run when the budget is n [Section 2.4]."""
     return list(range(warmup)) + list(range(n_layers - (n - warmup), n_layers))
@@ -218,6 +233,15 @@ class CachedDecoder:
         self.P = None
         self.k = self.v = None
         self.layer_steps = 0
+
+    def set_table(self, n_active, warmup):
+        """Installs an arbitrary non-increasing budget table."""
+        if any(b > a for a, b in zip(n_active, n_active[1:])) or any(not (warmup < n <= self.L) for n in n_active):
+            raise ValueError("budget table must be non-increasing with warmup < n <= n_layers")
+        self.n_active = list(n_active)
+        self.top_begin = [self.L - (n - warmup) for n in n_active]
+        self.warmup = warmup
+        return self.n_active, self.top_begin
 
     def set_schedule(self, max_layers, min_layers, warmup, gen_len):
         self.n_active, self.top_begin = schedule(max_layers, min_layers, warmup, gen_len, self.L)

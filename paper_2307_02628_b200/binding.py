@@ -20,7 +20,8 @@ SD_OK, SD_ERR_ARG, SD_ERR_STATE, SD_ERR_POSITION, SD_ERR_CAPACITY, SD_ERR_CUDA, 
 SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING, SD_OPT_PDL, SD_OPT_CLUSTER, SD_OPT_WEIGHT_TILES = 1, 2, 3, 4, 5, 6, 7
 KERNEL_CLASSES = ("embed", "layernorm", "gemm_qkv", "kv_append", "attention", "lm_head", "gemm_out", "gemm_fc1", "gemm_fc2")
 
-EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_layer_capacity",
+EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_schedule_power_compute",
+           "sd_schedule_custom", "sd_layer_capacity",
            "sd_prefill", "sd_decode_step", "sd_decode_step_static", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_status", "sd_stats",
            "sd_set_option", "sd_kernel_time", "sd_kernel_time_reset", "sd_strerror", "sd_destroy")
 
@@ -64,6 +65,8 @@ def lib() -> C.CDLL:
     L.sd_create.argtypes = [C.POINTER(SdConfig), C.POINTER(SdWeights), C.POINTER(SdPlan), vp, C.c_size_t, vp, C.POINTER(vp)]
     L.sd_schedule.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, i32p, i32p]
     L.sd_schedule_compute.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i32p, i32p]
+    L.sd_schedule_power_compute.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i32p, i32p]
+    L.sd_schedule_custom.argtypes = [vp, i32p, C.c_int, C.c_int, i32p]
     L.sd_layer_capacity.argtypes = [C.POINTER(SdConfig), C.POINTER(SdPlan), i32p]
     L.sd_prefill.argtypes = [vp, vp, C.c_int, C.c_int, vp]
     L.sd_decode_step.argtypes = [vp, vp, C.c_int, vp]
@@ -103,6 +106,15 @@ def schedule_compute(n_layers: int, max_layers: int, min_layers: int, warmup: in
     n = (C.c_int32 * max(gen_len, 1))()
     t = (C.c_int32 * max(gen_len, 1))()
     _check(lib().sd_schedule_compute(n_layers, max_layers, min_layers, warmup, gen_len, n, t), "sd_schedule_compute")
+    return list(n)[:gen_len], list(t)[:gen_len]
+
+
+def schedule_power_compute(n_layers: int, max_layers: int, min_layers: int, warmup: int, gen_len: int, alpha: int):
+    """Power-law budget table, host only: (n_active, top_begin) as lists."""
+    n = (C.c_int32 * max(gen_len, 1))()
+    t = (C.c_int32 * max(gen_len, 1))()
+    _check(lib().sd_schedule_power_compute(n_layers, max_layers, min_layers, warmup, gen_len, alpha, n, t),
+           "sd_schedule_power_compute")
     return list(n)[:gen_len], list(t)[:gen_len]
 
 
@@ -167,6 +179,13 @@ class Decoder:
         t = (C.c_int32 * max(gen_len, 1))()
         _check(lib().sd_schedule(self.h, max_layers, min_layers, warmup, gen_len, n, t), "sd_schedule")
         return list(n)[:gen_len], list(t)[:gen_len]
+
+    def schedule_custom(self, n_active, warmup: int):
+        G = len(n_active)
+        n = (C.c_int32 * G)(*n_active)
+        t = (C.c_int32 * G)()
+        _check(lib().sd_schedule_custom(self.h, n, warmup, G, t), "sd_schedule_custom")
+        return list(t)
 
     def prefill(self, tokens: torch.Tensor, logits: torch.Tensor | None = None) -> torch.Tensor:
         B, P = tokens.shape

@@ -102,6 +102,18 @@ int budget_at(int mx, int mn, int g, int G) {
   return mn + (int)((2 * (den - g) * D + den) / (2 * den));
 }
 
+// Power-law variant (Section 2.3 names it as another possible decay): min + (max - min) (1 - t)^alpha
+// with t = g / (G - 1) and an integer exponent, rounded to nearest with halves up, in integers:
+// min + floor((2 D (G-1-g)^alpha + (G-1)^alpha) / (2 (G-1)^alpha)).  alpha = 1 is the linear schedule.
+int budget_power_at(int mx, int mn, int g, int G, int alpha) {
+  if (G == 1) return mx;
+  const unsigned __int128 den1 = G - 1, num1 = G - 1 - g;
+  unsigned __int128 den = 1, num = 1;
+  for (int i = 0; i < alpha; ++i) { den *= den1; num *= num1; }
+  const unsigned __int128 D = mx - mn;
+  return mn + (int)((2 * D * num + den) / (2 * den));
+}
+
 // number of generated indices at which layer l runs under (mx, mn, w, G)
 void layer_counts(int L, int mx, int mn, int w, int G, std::vector<int>& count) {
   count.assign(L, 0);
@@ -548,6 +560,44 @@ int sd_schedule(sd_handle* h, int mx, int mn, int w, int G, int32_t* n_active, i
   h->warmup = w; h->gen_len = G;
   h->have_schedule = true;
   // the prompt's cache does not depend on the schedule: keep it when the new length still fits
+  if (h->have_prefill && (int64_t)h->P + G > h->cfg.max_pos) h->have_prefill = false;
+  h->next_pos = h->P;
+  return SD_OK;
+}
+
+int sd_schedule_power_compute(int n_layers, int mx, int mn, int w, int G, int alpha, int32_t* n_active, int32_t* top_begin) {
+  if (!valid_schedule_args(n_layers, mx, mn, w, G) || alpha < 1 || alpha > 8) return SD_ERR_ARG;
+  for (int g = 0; g < G; ++g) {
+    const int n = budget_power_at(mx, mn, g, G, alpha);
+    if (n_active) n_active[g] = n;
+    if (top_begin) top_begin[g] = n_layers - (n - w);
+  }
+  return SD_OK;
+}
+
+int sd_schedule_custom(sd_handle* h, const int32_t* n_active, int w, int G, int32_t* top_begin) {
+  if (!h || !n_active || G < 1 || G > h->cfg.max_gen || w < 0) return SD_ERR_ARG;
+  const int L = h->cfg.n_layers;
+  for (int g = 0; g < G; ++g) {
+    if (n_active[g] <= w || n_active[g] > L) return SD_ERR_ARG;
+    if (g > 0 && n_active[g] > n_active[g - 1]) return SD_ERR_ARG;      // budgets never grow (Section 2.2)
+  }
+  std::vector<int> count(L, 0);
+  for (int g = 0; g < G; ++g) {
+    const int top = L - (n_active[g] - w);
+    for (int l = 0; l < L; ++l)
+      if (l < w || l >= top) ++count[l];
+  }
+  for (int l = 0; l < L; ++l)
+    if (h->cfg.max_prompt + count[l] > h->A.cap[l]) return SD_ERR_CAPACITY;
+  h->n_active.assign(n_active, n_active + G);
+  h->top_begin.resize(G);
+  for (int g = 0; g < G; ++g) {
+    h->top_begin[g] = L - (n_active[g] - w);
+    if (top_begin) top_begin[g] = h->top_begin[g];
+  }
+  h->warmup = w; h->gen_len = G;
+  h->have_schedule = true;
   if (h->have_prefill && (int64_t)h->P + G > h->cfg.max_pos) h->have_prefill = false;
   h->next_pos = h->P;
   return SD_OK;

@@ -17,7 +17,7 @@ def make_decoder(wl: synth.Workload, weights, full_capacity=False, **kw):
                            full_capacity=full_capacity, **kw)
 
 
-def gpu_run_forced(dec, wl: synth.Workload, prompts, forced, rows=None):
+def gpu_run_forced(dec, wl: synth.Workload, prompts, forced, rows=None, table=None):
     """Prefill + gen_len decode steps feeding forced[:, g] at step g.
     Returns fp32 CPU logits [len(rows), gen_len + 1, vocab] (index 0 = prefill)."""
     B, G = wl.batch, wl.gen_len
@@ -25,7 +25,10 @@ def gpu_run_forced(dec, wl: synth.Workload, prompts, forced, rows=None):
     ridx = torch.tensor(rows, device=dec.device)
     out = torch.empty(len(rows), G + 1, wl.shape.vocab, dtype=torch.float32)
     with torch.cuda.stream(dec.stream):
-        dec.schedule(wl.max_layers, wl.min_layers, wl.warmup, G)
+        if table is None:
+            dec.schedule(wl.max_layers, wl.min_layers, wl.warmup, G)
+        else:
+            dec.schedule_custom(table, wl.warmup)       # caller-supplied budget per generated position
         logits = dec.prefill(prompts)
         out[:, 0] = logits[ridx].cpu()
         forced_d = forced.to(dec.device)
@@ -37,10 +40,10 @@ def gpu_run_forced(dec, wl: synth.Workload, prompts, forced, rows=None):
     return out
 
 
-def oracle_run_forced(wl: synth.Workload, weights, prompts, forced, rows=None, dtype=torch.float64):
+def oracle_run_forced(wl: synth.Workload, weights, prompts, forced, rows=None, dtype=torch.float64, table=None):
     """The definition on the same token sequences: logits [len(rows), gen_len + 1, vocab]."""
     rows = list(range(wl.batch)) if rows is None else rows
-    n, _ = O.schedule(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len, wl.shape.n_layers)
+    n = table if table is not None else O.schedule(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len, wl.shape.n_layers)[0]
     act = O.active_matrix(wl.shape.n_layers, wl.prompt_len, n, wl.warmup)
     seq = torch.cat([prompts, forced], dim=1)[rows]
     # the token fed at the last step produces logits for a position nobody consumes; keep it anyway

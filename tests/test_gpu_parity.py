@@ -260,3 +260,24 @@ def test_launch_modes_compute_the_same_function():
             for key, out in runs.items():
                 if key[0] == shape.name:
                     assert torch.equal(out, base), key
+
+
+@pytest.mark.parametrize("alpha", [2, 3])
+def test_power_law_budget_table(alpha):
+    """A caller-supplied budget table (power-law decay with warm-up 1) through sd_schedule_custom."""
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("toy-power", 6, 256, 4, 512, 999, 96, "bf16")
+    wl = synth.Workload(shape, 3, 21, 40, 6, 2, 1)
+    table, top = O.schedule_power(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len, shape.n_layers, alpha)
+    assert binding.schedule_power_compute(shape.n_layers, 6, 2, 1, 40, alpha) == (table, top)
+    w = synth.make_weights(shape, seed=13, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced, table=table)
+    dec = harness.make_decoder(wl, w)                       # cache plan: the linear 6 -> 2 schedule, which dominates
+    gpu = harness.gpu_run_forced(dec, wl, prompts, forced, table=table)
+    assert dec.stats() == (wl.gen_len, sum(table))
+    with pytest.raises(binding.SdError) as e:
+        dec.schedule_custom([2, 3] + [2] * 38, 1)           # a budget that grows is refused
+    assert e.value.code == binding.SD_ERR_ARG
+    dec.close()
+    _check(gpu, ref, "bf16", f"power law alpha={alpha}")

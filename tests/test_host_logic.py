@@ -71,3 +71,9 @@ def test_config_validation():
     with pytest.raises(binding.SdError):
         binding.arena_bytes(cfg, binding.SdPlan(4, 2, 0, 9, 0))     # plan longer than max_gen
     assert binding.lib().sd_strerror(binding.SD_ERR_POSITION).decode().startswith("position")
+
+
+@pytest.mark.parametrize("L,mx,mn,w,G,alpha", [(32, 32, 8, 0, 512, 1), (32, 32, 8, 0, 512, 2), (32, 22, 11, 1, 1024, 3),
+                                                 (24, 16, 8, 1, 2047, 4), (12, 12, 4, 0, 1, 2), (12, 12, 4, 0, 2, 8)])
+def test_power_law_schedule_is_bit_exact_with_the_oracle(L, mx, mn, w, G, alpha):
+    assert binding.schedule_power_compute(L, mx, mn, w, G, alpha) == tuple(O.schedule_power(mx, mn, w, G, L, alpha))

@@ -1,5 +1,6 @@
 """Pins for the oracle's schedule: what the paper prints and what arithmetic fixes."""
 import os
+import math
 from fractions import Fraction
 
 import pytest
@@ -111,3 +112,21 @@ def test_active_matrix_monotone_sets():
 def test_bad_arguments(args):
     with pytest.raises(ValueError):
         O.schedule(*args)
+
+
+@pytest.mark.parametrize("alpha", [1, 2, 3])
+def test_power_law_schedule(alpha):
+    L, mx, mn, w, G = 32, 22, 11, 1, 257
+    n, top = O.schedule_power(mx, mn, w, G, L, alpha)
+    lin, _ = O.schedule(mx, mn, w, G, L)
+    assert n[0] == mx and n[-1] == mn
+    assert all(a >= b for a, b in zip(n, n[1:]))
+    assert all(p <= q for p, q in zip(n, lin))               # (1 - t)^alpha <= 1 - t: never above the linear budget
+    if alpha == 1:
+        assert n == lin
+    else:
+        assert sum(n) < sum(lin)
+    # hand-checked point: t = 1/2 exactly at g = 128, line value min + D / 2^alpha
+    assert n[128] == math.floor(mn + Fraction(mx - mn, 2 ** alpha) + Fraction(1, 2))
+    for g, v in enumerate(n):
+        assert top[g] == L - (v - w)
