@@ -218,12 +218,14 @@ int sd_launch_count(sd_handle *h, int64_t *launches);
 enum {
   SD_OPT_GRAPHS = 1,       /* 1 (default): replay one CUDA graph per step shape; 0: plain launches */
   SD_OPT_ATTN_CHUNK = 2,   /* keys per split of the decode attention (multiple of 32); 0 = automatic */
-  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (128-row tensor-core kernel, else CUDA cores);
-                              1 = CUDA cores only; 2 = 128-row kernel; 3 = 256-row cluster kernel      */
+  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (token-stationary kernel up to 64 tokens, else the
+                              128-row weight-stationary kernel, else CUDA cores); 1 = CUDA cores only;
+                              2 = 128-row kernel; 3 = 256-row cluster kernel                           */
   SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
   SD_OPT_PDL = 5,          /* programmatic dependent launch: mask of kernel classes (1 << SD_K_*) whose
                               kernels may begin before their predecessor ends; 0 = none             */
-  SD_OPT_CLUSTER = 6,      /* blocks per cluster that split K in the 256-row GEMM: 0 = automatic, 1..4 */
+  SD_OPT_CLUSTER = 6,      /* blocks per cluster that split K in the cluster GEMMs: 0 = automatic, 1..4
+                              (the token-stationary kernel uses 1 or 2)                               */
   SD_OPT_WEIGHT_TILES = 7  /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
 };
 int sd_set_option(sd_handle *h, int option, int value);

@@ -15,6 +15,7 @@
 #include "kernels.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_wide.cuh"
+#include "gemm_xs.cuh"
 
 namespace {
 
@@ -68,6 +69,7 @@ struct sd_handle {
   int64_t k_launches[SD_K_COUNT] = {};
   sd::TcContext tc;
   sd::WideContext wide;
+  sd::XsContext xs;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(arena + off); }
   int* status() const { return at<int>(A.scalars); }
@@ -223,6 +225,7 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_of
   Lc.begin(cls);
   bool done = false;
   if (std::is_same<T, bf16>::value && h->opt_gemm != 1) {
+    if (h->opt_gemm == 0) done = sd::xs_gemm(h->xs, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp, h->wide.force_cluster);
     if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
     if (!done) done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
   }
@@ -253,6 +256,7 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
   h->tc.pdl = pdl_for(h, SD_K_GEMM_QKV);
   Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
+  if (h->opt_gemm == 0) done = sd::xs_gemm(h->xs, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp, h->wide.force_cluster);
   if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (done) Lc.end(); else Lc.cancel();
@@ -523,6 +527,7 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
   }
   sd::tc_init(h->tc);
   sd::wide_init(h->wide, h->tc);
+  sd::xs_init(h->xs, h->tc);
   if (h->tc.ready && h->A.packable) {            // tile-packed copies of the matrices, made once
     const int d = cfg->d_model, f = cfg->d_ffn;
     auto pack = [&](const void* W, size_t off, int n, int k) {

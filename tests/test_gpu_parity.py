@@ -209,7 +209,7 @@ def test_tensor_core_and_cuda_core_gemm_paths_agree(B, P):
     prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
     ref = harness.oracle_run_forced(wl, w, prompts, forced)
     outs = []
-    for mode in (1, 2, 0):          # CUDA cores, 128-row tcgen05 kernel, 256-row cluster kernel
+    for mode in (1, 2, 3, 0):       # CUDA cores, 128-row tcgen05 kernel, 256-row cluster kernel, automatic
         dec = harness.make_decoder(wl, w)
         dec.set_option(binding.SD_OPT_GEMM, mode)
         outs.append(harness.gpu_run_forced(dec, wl, prompts, forced))
@@ -218,6 +218,7 @@ def test_tensor_core_and_cuda_core_gemm_paths_agree(B, P):
     # a different summation order flips some bf16 roundings of the activations: ulp-scale differences
     assert float((outs[0] - outs[1]).abs().max()) < 1e-2
     assert float((outs[0] - outs[2]).abs().max()) < 1e-2
+    assert float((outs[0] - outs[3]).abs().max()) < 1e-2
 
 
 @pytest.mark.parametrize("cluster", [1, 2, 3, 4])
@@ -230,11 +231,15 @@ def test_cluster_split_k_reduce_scatter(cluster):
     w = synth.make_weights(shape, seed=10, random_ln=True)
     prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
     ref = harness.oracle_run_forced(wl, w, prompts, forced)
-    dec = harness.make_decoder(wl, w)
-    dec.set_option(binding.SD_OPT_CLUSTER, cluster)
-    out = harness.gpu_run_forced(dec, wl, prompts, forced)
-    dec.close()
-    _check(out, ref, "bf16", f"cluster {cluster}")
+    for mode in (3, 0):                 # 256-row weight-stationary kernel; token-stationary kernel (clusters of 1 or 2)
+        if mode == 0 and cluster > 2:
+            continue
+        dec = harness.make_decoder(wl, w)
+        dec.set_option(binding.SD_OPT_GEMM, mode)
+        dec.set_option(binding.SD_OPT_CLUSTER, cluster)
+        out = harness.gpu_run_forced(dec, wl, prompts, forced)
+        dec.close()
+        _check(out, ref, "bf16", f"gemm mode {mode} cluster {cluster}")
 
 
 def test_launch_modes_compute_the_same_function():
