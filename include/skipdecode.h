@@ -218,9 +218,10 @@ int sd_launch_count(sd_handle *h, int64_t *launches);
 enum {
   SD_OPT_GRAPHS = 1,       /* 1 (default): replay one CUDA graph per step shape; 0: plain launches */
   SD_OPT_ATTN_CHUNK = 2,   /* keys per split of the decode attention (multiple of 32); 0 = automatic */
-  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (token-stationary kernel up to 64 tokens, else the
-                              128-row weight-stationary kernel, else CUDA cores); 1 = CUDA cores only;
-                              2 = 128-row kernel; 3 = 256-row cluster kernel                           */
+  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (128-row weight-stationary tensor-core kernel, else
+                              CUDA cores); 1 = CUDA cores only; 2 = 128-row kernel; 3 = 256-row cluster
+                              kernel; 4 = token-stationary kernel (up to 64 tokens).  3 and 4 are measured
+                              alternatives that are slower at the shapes tried; they fall back to 2.    */
   SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
   SD_OPT_PDL = 5,          /* programmatic dependent launch: mask of kernel classes (1 << SD_K_*) whose
                               kernels may begin before their predecessor ends; 0 = none             */

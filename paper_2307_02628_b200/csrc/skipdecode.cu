@@ -225,7 +225,7 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_of
   Lc.begin(cls);
   bool done = false;
   if (std::is_same<T, bf16>::value && h->opt_gemm != 1) {
-    if (h->opt_gemm == 0) done = sd::xs_gemm(h->xs, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp, h->wide.force_cluster);
+    if (h->opt_gemm == 4) done = sd::xs_gemm(h->xs, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp, h->wide.force_cluster);
     if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
     if (!done) done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
   }
@@ -256,7 +256,7 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
   h->tc.pdl = pdl_for(h, SD_K_GEMM_QKV);
   Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
-  if (h->opt_gemm == 0) done = sd::xs_gemm(h->xs, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp, h->wide.force_cluster);
+  if (h->opt_gemm == 4) done = sd::xs_gemm(h->xs, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp, h->wide.force_cluster);
   if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (done) Lc.end(); else Lc.cancel();
@@ -733,7 +733,7 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != 0 && (value < kMinChunk || value % kMinChunk)) return SD_ERR_ARG;
       h->opt_chunk = value; return SD_OK;
     case SD_OPT_GEMM:
-      if (value < 0 || value > 3) return SD_ERR_ARG;
+      if (value < 0 || value > 4) return SD_ERR_ARG;
       if (value != h->opt_gemm) drop_graphs(h);
       h->opt_gemm = value; return SD_OK;
     case SD_OPT_CLUSTER:

@@ -209,7 +209,7 @@ def test_tensor_core_and_cuda_core_gemm_paths_agree(B, P):
     prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
     ref = harness.oracle_run_forced(wl, w, prompts, forced)
     outs = []
-    for mode in (1, 2, 3, 0):       # CUDA cores, 128-row tcgen05 kernel, 256-row cluster kernel, automatic
+    for mode in (1, 2, 3, 4):       # CUDA cores, 128-row tcgen05 kernel, 256-row cluster kernel, token-stationary kernel
         dec = harness.make_decoder(wl, w)
         dec.set_option(binding.SD_OPT_GEMM, mode)
         outs.append(harness.gpu_run_forced(dec, wl, prompts, forced))
@@ -231,8 +231,8 @@ def test_cluster_split_k_reduce_scatter(cluster):
     w = synth.make_weights(shape, seed=10, random_ln=True)
     prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
     ref = harness.oracle_run_forced(wl, w, prompts, forced)
-    for mode in (3, 0):                 # 256-row weight-stationary kernel; token-stationary kernel (clusters of 1 or 2)
-        if mode == 0 and cluster > 2:
+    for mode in (3, 4):                 # 256-row weight-stationary kernel; token-stationary kernel (clusters of 1 or 2)
+        if mode == 4 and cluster > 2:
             continue
         dec = harness.make_decoder(wl, w)
         dec.set_option(binding.SD_OPT_GEMM, mode)
