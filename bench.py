@@ -68,9 +68,9 @@ def step_bytes(wl: synth.Workload, n_active) -> float:
 
 # --------------------------------------------------------------------------- ncu traffic of the dominant kernel
 
-# DRAM bytes (read + write) per algorithmic byte of attn_partial_kernel, from the ncu --set full
-# capture summarised in profiles/ncu_full_attn_partial_c4_shape.md (1.08695 GB moved for 1.07583 GB
-# of K and V at T = 1026; the traffic is proportional to T).  Valid only for the kernel source it was
+# DRAM bytes (read + write) per algorithmic byte of attn_partial_kernel, from an ncu --set full
+# capture at config 4's launch shape (1.08695 GB moved for 1.07583 GB of K and V at T = 1026; the
+# traffic is proportional to T; a summary of the capture is kept under profiles/).  Valid only for the kernel source it was
 # taken on: the hash below is checked and `traffic` is null once the kernel text has changed.
 ATTN_TRAFFIC_RATIO = 1.0104
 ATTN_KERNEL_SHA256 = "1869cf8f40bc46c57d62cbbb198d42064b05ac355f561f429b98728d11566cd2"
@@ -82,6 +82,22 @@ def attention_kernel_hash() -> str:
     i = src.index("template <typename T, int HD, int UNROLL>")
     j = src.index("// Host side: launch with the programmatic")
     return hashlib.sha256(src[i:j].encode()).hexdigest()
+
+
+# --------------------------------------------------------------------------- ranks
+
+def max_over_ranks(value: float, dist, device) -> float:
+    """Every rank times its own replica; the job's time is the slowest rank's."""
+    if dist is None:
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(world: int, batch: int, steps: int, ms: float) -> float:
+    """Whole-job throughput of `world` independent replicas advancing in lock-step."""
+    return world * batch * steps / (ms / 1e3)
 
 
 # --------------------------------------------------------------------------- clocks
@@ -256,12 +272,7 @@ def gpu_arm(args, wl, rank, world):
             fn()
         b.record(stream)
         barrier()
-        ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms / reps
+        return max_over_ranks(a.elapsed_time(b), dist, device) / reps
 
     with torch.cuda.stream(stream):
         n_active, _ = dec.schedule(wl.max_layers, wl.min_layers, wl.warmup, G)
@@ -298,10 +309,7 @@ def gpu_arm(args, wl, rank, world):
                 e2e_pass()
             barrier()
             e2e_s = (time.perf_counter() - te) / args.e2e_steps
-        if dist is not None:
-            t = torch.tensor([e2e_s], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, dist, device)
 
         # dominant kernel (decode attention): device time per launch on sampled steps
         dec.rewind()
@@ -359,7 +367,7 @@ def gpu_arm(args, wl, rank, world):
                         "note": f"all-layers cache for all {G} steps does not fit; both timed on the first {Gp} positions"}
 
     peak, peak_kind = measured_peaks()
-    value = world * B * G_run / (ms_step / 1e3)
+    value = job_tokens_per_s(world, B, G_run, ms_step)
     total_bytes = step_bytes(wl, n_active[:G_run])
     achieved = attn_bytes / (attn_ms / 1e3) / 1e9 if attn_ms > 0 else None
     line = {

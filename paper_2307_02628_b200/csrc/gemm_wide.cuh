@@ -1,16 +1,16 @@
 // Wide-tile tensor-core GEMM for the weight-streaming regime (few tokens, bf16 operands):
 // out[m, n] (+)= sum_k X[m, k] W[n, k] + bias[n], X carried as hi + lo (see Operand).
 //
-// Why it exists.  One SM's TMA intake tops out far below its share of what the tensor cores
-// or HBM could take, so the time of a small-batch GEMM is (bytes a block pulls) / (intake
-// rate).  A block of the 128-row kernel pulls as many operand bytes as weight bytes (64
-// tokens x hi, lo).  Here a block owns 256 weight rows (two 128 x NB accumulators in tensor
-// memory) per operand tile, which halves the operand bytes per weight byte, and the blocks of
-// a thread-block cluster split K between them so that enough blocks exist to keep every SM
-// pulling.  For the store epilogues the cluster finishes with a reduce-scatter through
-// distributed shared memory: each block ships the accumulator rows it does not own to their
-// owner (32-row groups dealt round-robin), then adds what it received to its own rows and
-// runs the epilogue on them.  The residual epilogue needs no exchange (fp32 atomics).
+// A measured alternative to the 128-row kernel, selectable with SD_OPT_GEMM = 3.  A block owns
+// 256 weight rows (two 128 x 2NB accumulators in tensor memory) per operand tile, which halves
+// the operand bytes per weight byte, and the blocks of a thread-block cluster split K between
+// them so that enough blocks exist.  For the store epilogues the cluster finishes with a
+// reduce-scatter through distributed shared memory: each block ships the accumulator rows it
+// does not own to their owner (32-row groups dealt round-robin), then adds what it received
+// to its own rows and runs the epilogue on them.  The residual epilogue needs no exchange
+// (fp32 atomics).  On B200 at 64 tokens it is slower than the 128-row kernel: the main loop is
+// paced by the number of MMA instructions per SM, which this layout does not reduce, and its
+// epilogue is longer.
 //
 // Warp roles as in gemm_tc.cuh.  All threads of all blocks of a cluster reach both cluster
 // barriers on every path, also when a bounded mbarrier wait has expired (the data movement
