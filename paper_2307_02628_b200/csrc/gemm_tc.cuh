@@ -181,7 +181,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -264,7 +263,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         kv_base = n < 2 * qo.d ? qo.Kc : qo.Vc;
       }
     }
-    if (mbar_wait(accum_bar, 0, abort_flag, status)) {
+    const bool accum_ok = mbar_wait(accum_bar, 0, abort_flag, status);
+    // The main loop is over: let the next kernel of the stream become resident now, so that its
+    // launch and set-up overlap this kernel's epilogue (earlier would only park its blocks on the
+    // SMs for the whole main loop).
+    pdl_launch_dependents();
+    if (accum_ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const float b = (bias != nullptr && n < N && (EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
 #pragma unroll 1
