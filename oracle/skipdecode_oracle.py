@@ -27,6 +27,9 @@ What it computes (paper sections in brackets):
                         [Sections 2.1-2.3].
 * `full_forward`        an ordinary pre-LayerNorm OPT-style decoder with no notion
                         of skipping: the 1x base model of Section 3.1.
+* `sample_top_p`        the paper's token selection: temperature softmax, nucleus of
+                        mass top_p, inverse-CDF draw from a caller-supplied uniform
+                        number [Section 3.2: beam 1, top-p 0.7, temperature 0.3].
 
 Model (OPT-style, the family the paper evaluates in Section 3): learned absolute
 positions added to token embeddings; per layer  u = LN1(h);  q = (Wq u + bq)/sqrt(hd),
@@ -41,7 +44,10 @@ Table 2's budgets, exact rational arithmetic and the prose invariants;
 `forward_sequence` and `CachedDecoder` against each other, against `full_forward`
 for a full budget, against closed forms (bias-only model, zero-query attention =
 running mean of values, LayerNorm of a hand-computed vector) and against a
-scalar pure-Python evaluation on a toy model.
+scalar pure-Python evaluation on a toy model; `nucleus` / `sample_top_p` against an
+exhaustive search over all subsets of a small vocabulary, the Hugging Face
+temperature and top-p logits warpers, exact frequencies under equally spaced
+uniforms, and the argmax limits.
 Parity unpinned: absolute logit values with trained OPT weights and any output
 quality figure of the paper (no trained weights or datasets are available).
 """
@@ -306,3 +312,46 @@ class CachedDecoder:
 def greedy(logits: torch.Tensor) -> torch.Tensor:
     """Lowest index attaining the maximum of each row."""
     return torch.argmax(logits, dim=-1).to(torch.int32)
+
+
+# --------------------------------------------------------------------------- sampling
+
+def nucleus(logits_row: torch.Tensor, temperature: float, top_p: float):
+    """Temperature softmax and its nucleus for ONE row of logits.
+
+    The paper's generation settings are a beam of 1, top-p 0.7 and temperature 0.3
+    (Section 3.2, Datasets).  Top-p ("nucleus") sampling keeps the smallest set of
+    most probable tokens whose probabilities add up to at least top_p and samples
+    from that set in proportion to the probabilities.
+
+    Returns (order, probs, k): token ids sorted by decreasing probability (equal
+    probabilities: lower id first), their float64 probabilities in that order, and
+    the size k >= 1 of the nucleus, the first k entries of `order`.
+    """
+    x = logits_row.to(torch.float64) / float(temperature)
+    probs = torch.softmax(x, dim=0)
+    order = torch.sort(probs, descending=True, stable=True).indices
+    sorted_probs = probs[order]
+    cum = torch.cumsum(sorted_probs, dim=0)
+    reached = torch.nonzero(cum >= top_p)
+    k = int(reached[0]) + 1 if reached.numel() else int(probs.numel())
+    return order, sorted_probs, k
+
+
+def sample_top_p(logits: torch.Tensor, uniforms: torch.Tensor, temperature: float, top_p: float) -> torch.Tensor:
+    """One token per row by inverse-CDF sampling inside the nucleus.
+
+    `uniforms[b]` in [0, 1) is the random number of row b, supplied by the caller.
+    With the nucleus in decreasing-probability order and M its total probability,
+    the token chosen is the first whose running sum reaches uniforms[b] * M (the
+    last token of the nucleus if rounding leaves the target unreached).
+    """
+    out = torch.empty(logits.shape[0], dtype=torch.int32)
+    for b in range(logits.shape[0]):
+        order, sorted_probs, k = nucleus(logits[b], temperature, top_p)
+        cum = torch.cumsum(sorted_probs[:k], dim=0)
+        target = float(uniforms[b]) * float(cum[-1])
+        hit = torch.nonzero(cum > target)
+        j = int(hit[0]) if hit.numel() else k - 1
+        out[b] = int(order[j])
+    return out
