@@ -202,6 +202,19 @@ int sd_decode_step_host(sd_handle *h, const int32_t *h_token_ids, int position, 
  * d_logits: device fp32 [B, vocab]; d_next: device int32 [B]. */
 int sd_greedy(sd_handle *h, const float *d_logits, int B, int32_t *d_next);
 
+/* Sampled choice with the paper's generation settings (Section 3.2, Datasets: beam 1,
+ * top-p 0.7, temperature 0.3), any values accepted: p = softmax(d_logits[b, :] / temperature);
+ * the nucleus of row b is the smallest set of most probable tokens whose probabilities sum to
+ * at least top_p (equal probabilities: lower token id first); with the nucleus in order of
+ * decreasing probability and M its total probability, d_next[b] is the first token whose
+ * running sum exceeds d_uniforms[b] * M.  The random numbers are the caller's:
+ * d_uniforms: device fp32 [B], each in [0, 1) (values outside are clamped into the range).
+ * Probabilities are summed as 2^-40 fixed-point integers, so the result does not depend on
+ * thread order.  d_logits: device fp32 [B, vocab]; d_next: device int32 [B].
+ * Errors: SD_ERR_ARG unless temperature > 0 and 0 < top_p <= 1 (both finite). */
+int sd_sample_top_p(sd_handle *h, const float *d_logits, int B, float temperature, float top_p,
+                    const float *d_uniforms, int32_t *d_next);
+
 /* Synchronises the stream and reads the device status word (0 = no error; kernels
  * set bits on an out-of-range token id or a bounded wait that expired).
  * Returns SD_ERR_DEVICE when it is non-zero. */
@@ -227,7 +240,9 @@ enum {
                               kernels may begin before their predecessor ends; 0 = none             */
   SD_OPT_CLUSTER = 6,      /* blocks per cluster that split K in the cluster GEMMs: 0 = automatic, 1..4
                               (the token-stationary kernel uses 1 or 2)                               */
-  SD_OPT_WEIGHT_TILES = 7  /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
+  SD_OPT_WEIGHT_TILES = 7, /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
+  SD_OPT_PREFILL_ATTN = 8  /* 1 (default): sd_prefill's causal attention runs as 64x64 tensor-core tiles
+                              (bf16 storage, head size 64 or 128); 0: one decode-style block per query row */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff

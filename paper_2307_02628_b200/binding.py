@@ -17,12 +17,12 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libskipdec
 _lib = None
 
 SD_OK, SD_ERR_ARG, SD_ERR_STATE, SD_ERR_POSITION, SD_ERR_CAPACITY, SD_ERR_CUDA, SD_ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
-SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING, SD_OPT_PDL, SD_OPT_CLUSTER, SD_OPT_WEIGHT_TILES = 1, 2, 3, 4, 5, 6, 7
+SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING, SD_OPT_PDL, SD_OPT_CLUSTER, SD_OPT_WEIGHT_TILES, SD_OPT_PREFILL_ATTN = 1, 2, 3, 4, 5, 6, 7, 8
 KERNEL_CLASSES = ("embed", "layernorm", "gemm_qkv", "kv_append", "attention", "lm_head", "gemm_out", "gemm_fc1", "gemm_fc2")
 
 EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_schedule_power_compute",
            "sd_schedule_custom", "sd_layer_capacity",
-           "sd_prefill", "sd_decode_step", "sd_decode_step_static", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_status", "sd_stats",
+           "sd_prefill", "sd_decode_step", "sd_decode_step_static", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_sample_top_p", "sd_status", "sd_stats",
            "sd_set_option", "sd_kernel_time", "sd_kernel_time_reset", "sd_strerror", "sd_destroy")
 
 
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
     L.sd_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
     L.sd_decode_step_host.argtypes = [vp, vp, C.c_int, vp]
     L.sd_greedy.argtypes = [vp, vp, C.c_int, vp]
+    L.sd_sample_top_p.argtypes = [vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
     L.sd_status.argtypes = [vp, i32p]
     L.sd_stats.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
     L.sd_set_option.argtypes = [vp, C.c_int, C.c_int]
@@ -240,6 +241,17 @@ class Decoder:
         if out is None:
             out = torch.empty(B, dtype=torch.int32, device=self.device)
         _check(lib().sd_greedy(self.h, logits.data_ptr(), B, out.data_ptr()), "sd_greedy")
+        return out
+
+    def sample_top_p(self, logits: torch.Tensor, uniforms: torch.Tensor, temperature: float = 0.3,
+                     top_p: float = 0.7, out: torch.Tensor | None = None) -> torch.Tensor:
+        B = logits.shape[0]
+        if out is None:
+            out = torch.empty(B, dtype=torch.int32, device=self.device)
+        assert uniforms.dtype == torch.float32 and uniforms.is_cuda and uniforms.numel() == B
+        self._order()
+        _check(lib().sd_sample_top_p(self.h, logits.data_ptr(), B, temperature, top_p, uniforms.data_ptr(),
+                                     out.data_ptr()), "sd_sample_top_p")
         return out
 
     def status(self) -> int:

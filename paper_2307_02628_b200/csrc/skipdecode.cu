@@ -4,6 +4,7 @@
 #include "../../include/skipdecode.h"
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <map>
@@ -16,6 +17,8 @@
 #include "gemm_tc.cuh"
 #include "gemm_wide.cuh"
 #include "gemm_xs.cuh"
+#include "sample.cuh"
+#include "attn_prefill.cuh"
 
 namespace {
 
@@ -58,7 +61,7 @@ struct sd_handle {
   int B = 0, P = 0, next_pos = 0;
   int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
-  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = SD_PDL_DEFAULT, opt_tiles = 1;
+  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = SD_PDL_DEFAULT, opt_tiles = 1, opt_prefill = 1;
   bool packed = false;       // the arena holds tile-packed copies of the weight matrices
   // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
   struct Graph { cudaGraphExec_t exec; int64_t nodes; };
@@ -284,13 +287,43 @@ void launch_attention(Launcher& Lc, const T* Kc, const T* Vc, int cap, int rows,
   }
 }
 
+// Prompt pass, bf16 storage, head size 64 or 128: tensor-core tiles over whole sequences.
+template <int HD>
+bool launch_attention_prefill_hd(Launcher& Lc, const bf16* Kc, const bf16* Vc, int cap, int n_seq, int P, int b0) {
+  sd_handle* h = Lc.h;
+  constexpr int smem = 2 * 2 * sd::PF_BN * HD * 2;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(sd::attn_prefill_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    configured = true;
+  }
+  Lc.begin(SD_K_ATTENTION);
+  dim3 grid((P + sd::PF_BM - 1) / sd::PF_BM, n_seq * h->cfg.n_heads);
+  sd::launch_kernel(false, h->stream, sd::attn_prefill_kernel<HD>, grid, dim3(sd::PF_THREADS), smem, (const float*)h->at<float>(h->A.qkv),
+                    3 * h->cfg.d_model, Kc, Vc, cap, h->cfg.n_heads, P, b0, h->at<bf16>(h->A.o));
+  Lc.end();
+  return true;
+}
+template <typename T>
+bool launch_attention_prefill(Launcher& Lc, const T* Kc, const T* Vc, int cap, int n_seq, int P, int b0) {
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (!Lc.h->opt_prefill) return false;
+    if (Lc.h->hd == 128) return launch_attention_prefill_hd<128>(Lc, Kc, Vc, cap, n_seq, P, b0);
+    if (Lc.h->hd == 64) return launch_attention_prefill_hd<64>(Lc, Kc, Vc, cap, n_seq, P, b0);
+  }
+  return false;
+}
+
 int ln_threads(int d) { return std::max(32, std::min(256, (d / 4 + 31) / 32 * 32)); }
 
 // One decoder layer over `rows` query rows (Sections 2.1, 2.2): LN1 -> QKV -> append K,V at
 // the rows' positions -> attention over cache positions 0..pos -> out-proj (+residual) ->
 // LN2 -> fc1 + ReLU -> fc2 (+residual).
 template <typename T>
-void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int n_chunks) {
+void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int n_chunks, int prompt_len = 0) {
   sd_handle* h = Lc.h;
   const sd_config& c = h->cfg;
   const int d = c.d_model, f = c.d_ffn;
@@ -312,7 +345,9 @@ void enqueue_layer(Launcher& Lc, int l, int rows, sd::RowMap map, int chunk, int
     sd::launch_kernel(pdl_for(h, SD_K_KV_APPEND), h->stream, sd::kv_append_kernel<T>, dim3(rows), dim3(256), 0, qkv, Kc, Vc, d, c.n_heads, h->hd, cap, map);
     Lc.end();
   }
-  launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
+  // prompt_len > 0: the rows are whole sequences of that length (the prompt pass)
+  if (!(prompt_len > 0 && prompt_len <= cap && launch_attention_prefill<T>(Lc, Kc, Vc, cap, rows / prompt_len, prompt_len, map.b0)))
+    launch_attention<T>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks);
   launch_gemm<T>(Lc, SD_K_GEMM_OUT, o, (const T*)h->w_o[l], h->A.wp_o[l], (const T*)h->b_o[l], rows, d, d, x, d, sd::EPI_RESIDUAL_F32);
   Lc.begin(SD_K_LAYERNORM);
   sd::launch_kernel(pdl_for(h, SD_K_LAYERNORM), h->stream, sd::layernorm_kernel<T>, dim3(rows), dim3(ln_threads(d)), 0, x, (const T*)h->ln2_g[l], (const T*)h->ln2_b[l], u, d, c.ln_eps, nullptr);
@@ -390,7 +425,7 @@ int run_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_lo
     sd::RowMap map{P, b0, 0, nullptr};
     enqueue_embed<T>(Lc, d_tokens + (size_t)b0 * P, rows, map);
     const int chunk = (P + kMinChunk - 1) / kMinChunk * kMinChunk;   // one split: every row reads keys 0..pos
-    for (int l = 0; l < L; ++l) enqueue_layer<T>(Lc, l, rows, map, chunk, 1);
+    for (int l = 0; l < L; ++l) enqueue_layer<T>(Lc, l, rows, map, chunk, 1, P);
     last_rows_kernel<<<(nb + 127) / 128, 128, 0, h->stream>>>(h->at<int>(h->A.row_index), nb, P);
     enqueue_head<T>(Lc, nb, h->at<int>(h->A.row_index), d_logits + (size_t)b0 * h->cfg.vocab);
     Lc.count += 1;
@@ -709,6 +744,17 @@ int sd_greedy(sd_handle* h, const float* d_logits, int B, int32_t* d_next) {
   return cudaGetLastError() == cudaSuccess ? SD_OK : SD_ERR_CUDA;
 }
 
+int sd_sample_top_p(sd_handle* h, const float* d_logits, int B, float temperature, float top_p,
+                    const float* d_uniforms, int32_t* d_next) {
+  if (!h || !d_logits || !d_uniforms || !d_next || B < 1) return SD_ERR_ARG;
+  if (!std::isfinite(temperature) || !(temperature > 0.0f) || !std::isfinite(top_p) || !(top_p > 0.0f) || top_p > 1.0f)
+    return SD_ERR_ARG;
+  sd::sample_top_p_kernel<<<B, sd::SAMPLE_THREADS, 0, h->stream>>>(d_logits, h->cfg.vocab, d_uniforms,
+                                                                  1.0f / temperature, top_p, d_next);
+  h->launches += 1;
+  return cudaGetLastError() == cudaSuccess ? SD_OK : SD_ERR_CUDA;
+}
+
 int sd_status(sd_handle* h, int32_t* device_status) {
   if (!h) return SD_ERR_ARG;
   int32_t v = 0;
@@ -740,6 +786,8 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value < 0 || value > sd::tcw::MAX_CLUSTER) return SD_ERR_ARG;
       if (value != h->wide.force_cluster) drop_graphs(h);
       h->wide.force_cluster = value; return SD_OK;
+    case SD_OPT_PREFILL_ATTN:
+      h->opt_prefill = value ? 1 : 0; return SD_OK;
     case SD_OPT_WEIGHT_TILES:
       if ((value != 0) != (h->opt_tiles != 0)) drop_graphs(h);
       h->opt_tiles = value ? 1 : 0; return SD_OK;

@@ -170,3 +170,19 @@ def sample_rows(batch: int, count: int, seed: int = 2) -> list:
             break
         rows.add(r)
     return sorted(rows)
+
+
+def make_logits(batch: int, vocab: int, seed: int, scale: float = 1.0, step: float = 0.0) -> torch.Tensor:
+    """Stand-in logits for the token-selection tests: N(0, scale) fp32 [batch, vocab]; with
+    step > 0 they are rounded to multiples of `step`, which makes many of them equal."""
+    t = _normal(seed, f"logits:{batch}x{vocab}", (batch, vocab), scale, torch.float32)
+    if step > 0:
+        t = torch.round(t / step) * step
+    return t
+
+
+def make_uniforms(batch: int, seed: int) -> torch.Tensor:
+    """The random numbers of one sampling step: fp32 [batch] in [0, 1)."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(_seed_for(seed, f"uniforms:{batch}"))
+    return torch.rand(batch, generator=g, dtype=torch.float32)

@@ -106,6 +106,26 @@ def test_head_dims_and_storage_types(hd, dtype):
     _check(gpu, ref, dtype, f"toy hd={hd} {dtype}")
 
 
+@pytest.mark.parametrize("hd,P", [(64, 64), (64, 65), (64, 200), (128, 129), (128, 255)])
+def test_prompt_attention_tiles(hd, P):
+    # the prompt pass's tensor-core attention: several 64-key tiles, a ragged last tile, both head sizes;
+    # the decode steps that follow read what every prompt position wrote in every layer
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape(f"toy-prompt-{hd}", 3, 256, 256 // hd, 384, 777, 320, "bf16")
+    wl = synth.Workload(shape, 3, P, 12, 3, 2, 0)
+    w = synth.make_weights(shape, seed=8, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced)
+    runs = {}
+    for tiles in (1, 0):
+        dec = harness.make_decoder(wl, w)
+        dec.set_option(binding.SD_OPT_PREFILL_ATTN, tiles)
+        runs[tiles] = harness.gpu_run_forced(dec, wl, prompts, forced)
+        dec.close()
+        _check(runs[tiles], ref, "bf16", f"prompt attention hd={hd} P={P} tiles={tiles}")
+    assert float((runs[1] - runs[0]).abs().max()) <= 1e-2
+
+
 @pytest.mark.parametrize("chunk", [32, 64, 96])
 def test_attention_split_sizes_agree(chunk):
     from paper_2307_02628_b200 import binding
