@@ -27,6 +27,8 @@ What it computes (paper sections in brackets):
                         [Sections 2.1-2.3].
 * `full_forward`        an ordinary pre-LayerNorm OPT-style decoder with no notion
                         of skipping: the 1x base model of Section 3.1.
+* `forward_ragged`      rows of different prompt lengths in one batch, aligned at the
+                        right: each row alone, budgets taken by slot [Sections 2.1, 5].
 * `sample_top_p`        the paper's token selection: temperature softmax, nucleus of
                         mass top_p, inverse-CDF draw from a caller-supplied uniform
                         number [Section 3.2: beam 1, top-p 0.7, temperature 0.3].
@@ -210,6 +212,34 @@ def forward_sequence(weights: dict, n_heads: int, tokens: torch.Tensor, active: 
         h = torch.cat([_causal_layer(h[:, :m], weights["layers"][l], n_heads, dtype), h[:, m:]], dim=1)
     logits = _head(weights, h[:, logits_from:], dtype)
     return (logits, h) if return_hidden else logits
+
+
+def forward_ragged(weights: dict, n_heads: int, tokens: torch.Tensor, pad, active: torch.Tensor,
+                   dtype=torch.float64, logits_from: int = 0) -> torch.Tensor:
+    """Left-padded batch: row b's sequence occupies slots pad[b]..S-1 of tokens[b].
+
+    Batching puts every row's token of one step into the same slot, and the layer
+    budget belongs to the slot (all tokens of a batch at one position share it,
+    Section 2.1); rows of different prompt lengths are aligned at the right, so a
+    shorter row starts later (the limitation discussed in Section 5: rows can only
+    share a batch at matching positions).  Padding must be invisible: row b is the
+    sequence tokens[b, pad[b]:] on its own, its first real token at position 0,
+    with slot s using the layer set active[s].  Each row is therefore evaluated
+    alone by `forward_sequence`.  Returns logits [B, S - logits_from, V]; entries
+    of slots that hold padding are NaN.
+    """
+    B, S = tokens.shape
+    out = None
+    for b in range(B):
+        p = int(pad[b])
+        if not 0 <= p < S:
+            raise ValueError("a row needs at least one real token")
+        lg = forward_sequence(weights, n_heads, tokens[b:b + 1, p:], active[p:], dtype,
+                              logits_from=max(logits_from - p, 0))[0]
+        if out is None:
+            out = torch.full((B, S - logits_from, lg.shape[-1]), float("nan"), dtype=lg.dtype)
+        out[b, S - logits_from - lg.shape[0]:] = lg
+    return out
 
 
 def full_forward(weights: dict, n_heads: int, tokens: torch.Tensor, dtype=torch.float64) -> torch.Tensor:

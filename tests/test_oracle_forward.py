@@ -27,7 +27,7 @@ def toy_weights(shape, seed=7, std=0.3):
     return w
 
 
-def hf_logits(shape, w, tokens):
+def hf_logits(shape, w, tokens, attention_mask=None):
     from transformers import OPTConfig, OPTForCausalLM
     cfg = OPTConfig(vocab_size=shape.vocab, hidden_size=shape.d_model, num_hidden_layers=shape.n_layers,
                     ffn_dim=shape.d_ffn, num_attention_heads=shape.n_heads,
@@ -64,6 +64,8 @@ def hf_logits(shape, w, tokens):
     missing, unexpected = m.load_state_dict({k: v.double() for k, v in sd.items()}, strict=False)
     assert not unexpected and all("lm_head" in k for k in missing), (missing, unexpected)
     with torch.no_grad():
+        if attention_mask is not None:
+            return m(tokens.long(), attention_mask=attention_mask.long()).logits
         return m(tokens.long()).logits
 
 
@@ -327,3 +329,47 @@ def test_planted_mistakes_are_caught(monkeypatch, mistake):
         monkeypatch.setattr(torch, "triu", lambda x, diagonal=0: torch.zeros_like(x))
     gap, _ = hf_gap()
     assert gap > 1e-4, (mistake, gap)
+
+
+# ---------------------------------------------------------------- ragged (left-padded) batches
+
+def test_ragged_rows_match_library_opt_with_a_left_padded_mask():
+    # the library model given a left-padded batch and its attention mask (positions counted from each
+    # row's first real token) against the oracle's rows-on-their-own evaluation, full budget
+    shape = toy_shape()
+    w = toy_weights(shape)
+    S, pad = 13, [0, 4, 9, 12]
+    tokens = synth.make_tokens(shape.vocab, len(pad), S, seed=9)
+    mask = torch.ones(len(pad), S, dtype=torch.long)
+    for b, p in enumerate(pad):
+        mask[b, :p] = 0
+    ref = hf_logits(shape, w, tokens, attention_mask=mask)
+    active = torch.ones(S, shape.n_layers, dtype=torch.bool)
+    got = O.forward_ragged(w, shape.n_heads, tokens, pad, active, F64)
+    for b, p in enumerate(pad):
+        assert torch.isnan(got[b, :p]).all()
+        assert float((got[b, p:] - ref[b, p:]).abs().max()) < 1e-9
+    # and the pad tokens' identities are irrelevant
+    other = tokens.clone()
+    other[2, :9] = (other[2, :9] + 7) % shape.vocab
+    again = O.forward_ragged(w, shape.n_heads, other, pad, active, F64)
+    assert torch.equal(again[2, 9:], got[2, 9:])
+
+
+def test_ragged_budget_goes_by_slot_not_by_row_position():
+    # a row that starts late takes the layer set of the slot it sits in: with pad 0 the ragged evaluation
+    # is the plain one, and a padded row equals the plain evaluation of its tokens under the shifted table
+    shape = toy_shape(L=4)
+    w = toy_weights(shape, seed=3)
+    P, G = 6, 7
+    n, _ = O.schedule(4, 1, 0, G, 4)
+    active = O.active_matrix(4, P, n, 0)
+    tokens = synth.make_tokens(shape.vocab, 2, P + G, seed=2)
+    rag = O.forward_ragged(w, shape.n_heads, tokens, [0, 3], active, F64)
+    plain = O.forward_sequence(w, shape.n_heads, tokens, active, F64)
+    assert torch.equal(rag[0], plain[0])
+    alone = O.forward_sequence(w, shape.n_heads, tokens[1:2, 3:], active[3:], F64)[0]
+    assert torch.equal(rag[1, 3:], alone)
+    # the shifted row really differs from running it with the unshifted table
+    unshifted = O.forward_sequence(w, shape.n_heads, tokens[1:2, 3:], active[:P + G - 3], F64)[0]
+    assert float((unshifted - alone).abs().max()) > 1e-6
