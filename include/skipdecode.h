@@ -188,6 +188,27 @@ int sd_decode_step(sd_handle *h, const int32_t *d_token_ids, int position, float
 #define SD_STATIC_SCRATCH_BYTES (16u << 20)
 int sd_decode_step_static(sd_handle *h, const int32_t *d_token_ids, int position, float *d_logits);
 
+/* Ragged batches (the batching limitation of Section 5: rows share a batch only at
+ * matching positions, so prompts of different lengths are aligned at the right).
+ *
+ * sd_set_padding, before sd_prefill: h_pad (HOST, int32 [B]) gives each row's number of
+ * left-padding slots, 0 <= h_pad[b] < P.  Row b's own sequence is d_tokens[b, h_pad[b]..P-1]:
+ * its first real token takes learned position 0, it never attends to a slot before
+ * h_pad[b], and what sits in the padding slots (any valid token id) has no effect on it.
+ * The layer budget of a step still goes by the slot, the same for every row (Section
+ * 2.1).  NULL removes the padding.  Either way the next call must be sd_prefill.
+ *
+ * sd_set_rows, after sd_prefill: h_rows (HOST, int32 [n], strictly increasing, each in
+ * [0, B)) lists the rows that still generate, e.g. after the others emitted their end
+ * token.  From then on sd_decode_step takes d_token_ids [n] and writes d_logits [n, vocab]
+ * for exactly those rows, in that order, at a cost of n rows; the other rows' cache
+ * entries are left as they are.  NULL restores all B rows; sd_prefill does too.
+ * Both calls copy their array before returning and synchronise the stream.
+ * Errors: SD_ERR_ARG (range, order, B mismatch at sd_prefill), SD_ERR_STATE (sd_set_rows
+ * before sd_prefill). */
+int sd_set_padding(sd_handle *h, const int32_t *h_pad, int B);
+int sd_set_rows(sd_handle *h, const int32_t *h_rows, int n);
+
 /* Restarts generation at the end of the prompt: the next sd_decode_step must be at
  * position P again.  The prompt's cache entries are kept; entries of generated
  * positions are overwritten as the new steps reach them.  Errors: SD_ERR_STATE. */

@@ -22,7 +22,7 @@ KERNEL_CLASSES = ("embed", "layernorm", "gemm_qkv", "kv_append", "attention", "l
 
 EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_schedule_power_compute",
            "sd_schedule_custom", "sd_layer_capacity",
-           "sd_prefill", "sd_decode_step", "sd_decode_step_static", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_sample_top_p", "sd_status", "sd_stats",
+           "sd_prefill", "sd_decode_step", "sd_decode_step_static", "sd_rewind", "sd_launch_count", "sd_decode_step_host", "sd_greedy", "sd_sample_top_p", "sd_set_padding", "sd_set_rows", "sd_status", "sd_stats",
            "sd_set_option", "sd_kernel_time", "sd_kernel_time_reset", "sd_strerror", "sd_destroy")
 
 
@@ -75,6 +75,8 @@ def lib() -> C.CDLL:
     L.sd_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
     L.sd_decode_step_host.argtypes = [vp, vp, C.c_int, vp]
     L.sd_greedy.argtypes = [vp, vp, C.c_int, vp]
+    L.sd_set_padding.argtypes = [vp, vp, C.c_int]
+    L.sd_set_rows.argtypes = [vp, vp, C.c_int]
     L.sd_sample_top_p.argtypes = [vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
     L.sd_status.argtypes = [vp, i32p]
     L.sd_stats.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
@@ -197,10 +199,13 @@ class Decoder:
         _check(lib().sd_prefill(self.h, tokens.data_ptr(), B, P, logits.data_ptr()), "sd_prefill")
         self._keep_io = (tokens, logits)
         self.B, self.P = B, P
+        self._n_rows = None
         return logits
 
     def decode_step(self, ids: torch.Tensor, position: int, logits: torch.Tensor | None = None) -> torch.Tensor:
         ids = self._dev_i32(ids)
+        n = getattr(self, "_n_rows", None) or self.B
+        assert ids.numel() == n, f"{ids.numel()} token ids for {n} generating rows"
         if logits is None:
             logits = torch.empty(ids.shape[0], self.shape.vocab, dtype=torch.float32, device=self.device)
         self._order()
@@ -242,6 +247,24 @@ class Decoder:
             out = torch.empty(B, dtype=torch.int32, device=self.device)
         _check(lib().sd_greedy(self.h, logits.data_ptr(), B, out.data_ptr()), "sd_greedy")
         return out
+
+    def set_padding(self, pad=None):
+        """Left-padding slots per row (host list), or None to remove; call before prefill."""
+        if pad is None:
+            _check(lib().sd_set_padding(self.h, None, 0), "sd_set_padding")
+            return
+        arr = (C.c_int32 * len(pad))(*[int(p) for p in pad])
+        _check(lib().sd_set_padding(self.h, arr, len(pad)), "sd_set_padding")
+
+    def set_rows(self, rows=None):
+        """Rows that still generate (host list, increasing), or None for all; call after prefill."""
+        if rows is None:
+            _check(lib().sd_set_rows(self.h, None, 0), "sd_set_rows")
+            self._n_rows = None
+            return
+        arr = (C.c_int32 * len(rows))(*[int(r) for r in rows])
+        _check(lib().sd_set_rows(self.h, arr, len(rows)), "sd_set_rows")
+        self._n_rows = len(rows)
 
     def sample_top_p(self, logits: torch.Tensor, uniforms: torch.Tensor, temperature: float = 0.3,
                      top_p: float = 0.7, out: torch.Tensor | None = None) -> torch.Tensor:

@@ -50,11 +50,13 @@ __device__ __forceinline__ void pf_split(float x, float y, uint32_t& hi, uint32_
 // qkv: fp32 [n_seq * P, ldq], q of head h at columns h*HD..; row = seq * P + pos.
 // Kc, Vc: bf16 [B, H, cap, HD] of this layer; sequences b0.. of the batch.
 // o: bf16 operand rows [n_seq * P, 2 * H * HD] (hi | lo).
+// pad (may be null): left-padding slots per batch row; a row's keys start at slot pad[b], and a
+// padding slot attends to itself alone (its output is never used).
 template <int HD>
 __global__ void __launch_bounds__(PF_THREADS)
 attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16* __restrict__ Kc,
                     const __nv_bfloat16* __restrict__ Vc, int cap, int H, int P, int b0,
-                    __nv_bfloat16* __restrict__ o) {
+                    const int* __restrict__ pad, __nv_bfloat16* __restrict__ o) {
   constexpr int ROW_BYTES = HD * 2, CHUNKS = HD / 8;            // 16-byte chunks per key row
   constexpr int TILE_BYTES = PF_BN * ROW_BYTES;
   constexpr int KS = HD / 16;                                  // k-steps of Q K^T
@@ -67,7 +69,9 @@ attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16*
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int q0 = qt * PF_BM + warp * 16;                        // first query position of this warp
-  const int n_kt = qt + 1;                                     // key tiles 0..qt (the last one is masked)
+  const int n_kt = qt + 1;                                     // key tiles ..qt (the last one is masked)
+  const int first = pad ? pad[b0 + seq] : 0;                   // first slot of this row's own sequence
+  const int kt0 = min(first, qt * PF_BM) / PF_BN;              // tiles wholly inside the padding are skipped
 
   const size_t head_base = ((size_t)(b0 + seq) * H + h) * (size_t)cap * HD;
   const __nv_bfloat16* Kh = Kc + head_base;
@@ -87,7 +91,7 @@ attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16*
     }
   };
 
-  load_tile(0, 0);
+  load_tile(kt0, kt0 & 1);
   pf_commit();
 
   // q of this warp's 16 rows as MMA A fragments, scaled by hd^-1/2 log2(e), split into hi and lo
@@ -116,7 +120,7 @@ attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16*
 
   const int mi = lane >> 3, mr = lane & 7;                     // matrix and row this lane addresses in an x4 load
 
-  for (int kt = 0; kt < n_kt; ++kt) {
+  for (int kt = kt0; kt < n_kt; ++kt) {
     const int stage = kt & 1;
     if (kt + 1 < n_kt) { load_tile(kt + 1, stage ^ 1); pf_commit(); pf_wait<1>(); }
     else pf_wait<0>();
@@ -141,16 +145,18 @@ attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16*
         pf_mma(s[2 * np + 1], ql[ks], b[2], b[3]);
       }
     }
-    // causal mask: only the last tile holds keys beyond a query's own position
-    if (kt == n_kt - 1) {
+    // causal mask: only the last tile holds keys beyond a query's own position; padding mask: only
+    // tiles that begin before the row's first slot hold keys it must not see
+    if (kt == n_kt - 1 || kt * PF_BN < first) {
       const int p_lo = q0 + g, p_hi = p_lo + 8;
+      const int f_lo = min(first, p_lo), f_hi = min(first, p_hi);
 #pragma unroll
       for (int n = 0; n < NT_S; ++n) {
         const int j = kt * PF_BN + n * 8 + 2 * t;
-        if (j > p_lo) s[n][0] = -INFINITY;
-        if (j + 1 > p_lo) s[n][1] = -INFINITY;
-        if (j > p_hi) s[n][2] = -INFINITY;
-        if (j + 1 > p_hi) s[n][3] = -INFINITY;
+        if (j > p_lo || j < f_lo) s[n][0] = -INFINITY;
+        if (j + 1 > p_lo || j + 1 < f_lo) s[n][1] = -INFINITY;
+        if (j > p_hi || j < f_hi) s[n][2] = -INFINITY;
+        if (j + 1 > p_hi || j + 1 < f_hi) s[n][3] = -INFINITY;
       }
     }
     // online softmax (base 2); a row's values sit in the four lanes of a quad
@@ -164,10 +170,13 @@ attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16*
     mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-    // key 0 is visible to every query, so the maxima are finite from the first tile on
+    // a row may have seen no key yet (tiles before its first slot): its maximum is still -inf, every
+    // weight of the tile is 0, and the reference point of the exponentials is set to 0 to keep them finite
     const float sc_lo = m_lo == -INFINITY ? 0.f : exp2f(m_lo - mx_lo);
     const float sc_hi = m_hi == -INFINITY ? 0.f : exp2f(m_hi - mx_hi);
     m_lo = mx_lo; m_hi = mx_hi;
+    if (mx_lo == -INFINITY) mx_lo = 0.f;
+    if (mx_hi == -INFINITY) mx_hi = 0.f;
     l_lo *= sc_lo; l_hi *= sc_hi;
 #pragma unroll
     for (int n = 0; n < NT_O; ++n) { acc[n][0] *= sc_lo; acc[n][1] *= sc_lo; acc[n][2] *= sc_hi; acc[n][3] *= sc_hi; }

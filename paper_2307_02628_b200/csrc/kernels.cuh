@@ -91,16 +91,24 @@ __device__ __forceinline__ float block_sum(float v, float* scratch) {
   return scratch[32];
 }
 
-// Row r of a launch covers batch row b = b0 + r / q_per_b at position pos0 + r % q_per_b.
-// d_pos, when not null, supplies pos0 from device memory (graph replay).
+// Row r of a launch covers batch row b = b0 + r / q_per_b at position (cache slot)
+// pos0 + r % q_per_b.  d_pos, when not null, supplies pos0 from device memory (graph replay).
+// rows, when not null (decode steps, q_per_b = 1), lists the batch rows still generating:
+// b = rows[r].  pad, when not null, holds each batch row's number of left-padding slots: the
+// row's sequence starts at slot pad[b], so its learned position is pos - pad[b] and it
+// attends to slots pad[b]..pos only (a padding slot attends to itself alone).
 struct RowMap {
   int q_per_b, b0, pos0;
   const int* d_pos;
+  const int* rows;
+  const int* pad;
   __device__ __forceinline__ void get(int r, int& b, int& pos) const {
     const int p0 = d_pos ? *d_pos : pos0;
-    b = b0 + r / q_per_b;
+    b = rows ? rows[r] : b0 + r / q_per_b;
     pos = p0 + r % q_per_b;
   }
+  __device__ __forceinline__ int first_key(int b, int pos) const { return pad ? min(pad[b], pos) : 0; }
+  __device__ __forceinline__ int seq_pos(int b, int pos) const { return pad ? max(pos - pad[b], 0) : pos; }
 };
 
 // x[r, :] = tok_emb[ids[r], :] + pos_emb[pos(r), :]      (fp32 residual stream)
@@ -112,6 +120,7 @@ __global__ void embed_pos_kernel(const int32_t* __restrict__ ids, const T* __res
   const int r = blockIdx.x;
   int b, pos;
   map.get(r, b, pos);
+  pos = map.seq_pos(b, pos);
   int id = ids[r];
   if (id < 0 || id >= vocab || pos < 0 || pos >= max_pos) {   // record and clamp: never read out of range
     if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_TOKEN);
@@ -234,9 +243,11 @@ attn_partial_kernel(const float* __restrict__ qkv, int ldq, const T* __restrict_
   int b, pos;
   map.get(r, b, pos);
   const int T_len = min(pos + 1, cap);
-  const int k0 = blockIdx.y * chunk;
-  if (k0 >= T_len) return;
-  const int k1 = min(k0 + chunk, T_len);
+  if ((int)blockIdx.y * chunk >= T_len) return;
+  const int k1 = min((int)blockIdx.y * chunk + chunk, T_len);
+  // left padding: keys before the row's first slot do not exist for it.  A chunk that lies wholly
+  // in the padding walks no keys and publishes an empty partial (max -inf, sum 0).
+  const int k0 = max((int)blockIdx.y * chunk, map.first_key(b, pos));
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = lane / LPK, sub = lane % LPK;

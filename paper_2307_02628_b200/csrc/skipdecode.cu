@@ -36,7 +36,7 @@ struct Arena {            // byte offsets into the caller's arena
   size_t wp_head;
   bool packable;
   std::vector<int> cap;
-  size_t x, u, qkv, o, y, part_acc, part_ml, counters, row_index, ids, logits, scalars, total;
+  size_t x, u, qkv, o, y, part_acc, part_ml, counters, row_index, ids, logits, scalars, pad, rows, total;
   int rows_max;
   size_t part_slots;
 };
@@ -59,6 +59,12 @@ struct sd_handle {
   int warmup = 0, gen_len = 0;
   bool have_schedule = false, have_prefill = false;
   int B = 0, P = 0, next_pos = 0;
+  // ragged batches: left padding per row (host copy; device copy in the arena) and the rows still generating
+  std::vector<int> pad, rows;
+  bool have_pad = false, have_rows = false;
+  int n_rows() const { return have_rows ? (int)rows.size() : B; }
+  const int* d_pad() const { return have_pad ? at<int>(A.pad) : nullptr; }
+  const int* d_rows() const { return have_rows ? at<int>(A.rows) : nullptr; }
   int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
   int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = SD_PDL_DEFAULT, opt_tiles = 1, opt_prefill = 1;
@@ -178,6 +184,8 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   A.ids = take((size_t)c.max_batch * 4);
   A.logits = take((size_t)c.max_batch * c.vocab * 4);
   A.scalars = take(256);
+  A.pad = take((size_t)c.max_batch * 4);     // left-padding slots per batch row (ragged prompts)
+  A.rows = take((size_t)c.max_batch * 4);    // batch rows still generating
   A.total = off;
 }
 
@@ -303,7 +311,7 @@ bool launch_attention_prefill_hd(Launcher& Lc, const bf16* Kc, const bf16* Vc, i
   Lc.begin(SD_K_ATTENTION);
   dim3 grid((P + sd::PF_BM - 1) / sd::PF_BM, n_seq * h->cfg.n_heads);
   sd::launch_kernel(false, h->stream, sd::attn_prefill_kernel<HD>, grid, dim3(sd::PF_THREADS), smem, (const float*)h->at<float>(h->A.qkv),
-                    3 * h->cfg.d_model, Kc, Vc, cap, h->cfg.n_heads, P, b0, h->at<bf16>(h->A.o));
+                    3 * h->cfg.d_model, Kc, Vc, cap, h->cfg.n_heads, P, b0, h->d_pad(), h->at<bf16>(h->A.o));
   Lc.end();
   return true;
 }
@@ -404,13 +412,14 @@ int enqueue_decode(sd_handle* h, const int32_t* d_ids, int pos, bool pos_from_de
                    int n_chunks, bool timing, int64_t* launched, float* part_acc = nullptr, float* part_ml = nullptr) {
   Launcher Lc{h, timing, part_acc ? part_acc : h->at<float>(h->A.part_acc), part_ml ? part_ml : h->at<float>(h->A.part_ml)};
   const int L = h->cfg.n_layers, w = h->warmup, top = L - (n - w);
-  sd::RowMap map{1, 0, pos, pos_from_device ? h->d_pos() : nullptr};
-  enqueue_embed<T>(Lc, d_ids, h->B, map);
+  sd::RowMap map{1, 0, pos, pos_from_device ? h->d_pos() : nullptr, h->d_rows(), h->d_pad()};
+  const int rows = h->n_rows();
+  enqueue_embed<T>(Lc, d_ids, rows, map);
   for (int l = 0; l < L; ++l) {
     if (!(l < w || l >= top)) continue;             // bypassed layer: identity, no K/V written (Section 2.4)
-    enqueue_layer<T>(Lc, l, h->B, map, chunk, n_chunks);
+    enqueue_layer<T>(Lc, l, rows, map, chunk, n_chunks);
   }
-  enqueue_head<T>(Lc, h->B, nullptr, d_logits);
+  enqueue_head<T>(Lc, rows, nullptr, d_logits);
   *launched = Lc.count;
   return Lc.err;
 }
@@ -422,7 +431,7 @@ int run_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_lo
   const int per = std::max(1, kPrefillTokens / P);
   for (int b0 = 0; b0 < B; b0 += per) {
     const int nb = std::min(per, B - b0), rows = nb * P;
-    sd::RowMap map{P, b0, 0, nullptr};
+    sd::RowMap map{P, b0, 0, nullptr, nullptr, h->d_pad()};
     enqueue_embed<T>(Lc, d_tokens + (size_t)b0 * P, rows, map);
     const int chunk = (P + kMinChunk - 1) / kMinChunk * kMinChunk;   // one split: every row reads keys 0..pos
     for (int l = 0; l < L; ++l) enqueue_layer<T>(Lc, l, rows, map, chunk, 1, P);
@@ -457,7 +466,7 @@ int decode_step_impl(sd_handle* h, const int32_t* d_ids, int position, float* d_
   if (position != h->next_pos || g < 0 || g >= h->gen_len || position >= h->cfg.max_pos) return SD_ERR_POSITION;
   const int n = h->n_active[g];
   const int T = position + 1;
-  const int chunk = pick_chunk(h, h->B, T);
+  const int chunk = pick_chunk(h, h->n_rows(), T);
   const int n_chunks = (T + chunk - 1) / chunk;
   const bool bf = h->cfg.dtype == SD_DTYPE_BF16;
   int err = 0;
@@ -467,7 +476,7 @@ int decode_step_impl(sd_handle* h, const int32_t* d_ids, int position, float* d_
     err = bf ? enqueue_decode<bf16>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0, &launched)
              : enqueue_decode<float>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0, &launched);
   } else {
-    auto key = std::make_tuple(h->B, n, h->warmup, chunk, n_chunks, (const void*)d_ids, (const void*)d_logits);
+    auto key = std::make_tuple(h->n_rows(), n, h->warmup, chunk, n_chunks, (const void*)d_ids, (const void*)d_logits);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
       if (h->graphs.size() >= 256) drop_graphs(h);
@@ -665,10 +674,54 @@ int sd_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_log
   if (!h || !d_tokens || !d_logits || B < 1 || P < 1) return SD_ERR_ARG;
   if (!h->have_schedule) return SD_ERR_STATE;
   if (B > h->cfg.max_batch || P > h->cfg.max_prompt || (int64_t)P + h->gen_len > h->cfg.max_pos) return SD_ERR_CAPACITY;
+  if (h->have_pad) {                        // every row keeps at least one real token
+    if ((int)h->pad.size() != B) return SD_ERR_ARG;
+    for (int b = 0; b < B; ++b)
+      if (h->pad[b] >= P) return SD_ERR_ARG;
+  }
+  if (h->have_rows) { h->have_rows = false; h->rows.clear(); drop_graphs(h); }   // a new batch: all rows generate
   const int err = h->cfg.dtype == SD_DTYPE_BF16 ? run_prefill<bf16>(h, d_tokens, B, P, d_logits)
                                                 : run_prefill<float>(h, d_tokens, B, P, d_logits);
   if (err) return err;
   h->B = B; h->P = P; h->next_pos = P; h->have_prefill = true;
+  return SD_OK;
+}
+
+int sd_set_padding(sd_handle* h, const int32_t* h_pad, int B) {
+  if (!h) return SD_ERR_ARG;
+  if (!h_pad) {
+    if (h->have_pad) drop_graphs(h);
+    h->have_pad = false; h->pad.clear(); h->have_prefill = false;
+    return SD_OK;
+  }
+  if (B < 1 || B > h->cfg.max_batch) return SD_ERR_ARG;
+  for (int b = 0; b < B; ++b)
+    if (h_pad[b] < 0 || h_pad[b] >= h->cfg.max_prompt) return SD_ERR_ARG;
+  if (!h->have_pad) drop_graphs(h);
+  h->pad.assign(h_pad, h_pad + B);
+  h->have_pad = true;
+  h->have_prefill = false;                  // the cache was filled under another alignment
+  if (cudaMemcpyAsync(h->arena + h->A.pad, h->pad.data(), (size_t)B * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  return SD_OK;
+}
+
+int sd_set_rows(sd_handle* h, const int32_t* h_rows, int n) {
+  if (!h) return SD_ERR_ARG;
+  if (!h->have_prefill) return SD_ERR_STATE;
+  if (!h_rows) {
+    if (h->have_rows) drop_graphs(h);
+    h->have_rows = false; h->rows.clear();
+    return SD_OK;
+  }
+  if (n < 1 || n > h->B) return SD_ERR_ARG;
+  for (int i = 0; i < n; ++i)
+    if (h_rows[i] < 0 || h_rows[i] >= h->B || (i && h_rows[i] <= h_rows[i - 1])) return SD_ERR_ARG;
+  if (!h->have_rows) drop_graphs(h);
+  h->rows.assign(h_rows, h_rows + n);
+  h->have_rows = true;
+  if (cudaMemcpyAsync(h->arena + h->A.rows, h->rows.data(), (size_t)n * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
   return SD_OK;
 }
 
@@ -700,9 +753,9 @@ int sd_decode_step_static(sd_handle* h, const int32_t* d_ids, int position, floa
   if (attr.device != device) return SD_ERR_ARG;       // the static array of another GPU would be handed to this handle's kernels
   const int n = h->n_active[g];
   const int T = position + 1;
-  const int chunk = pick_chunk(h, h->B, T);
+  const int chunk = pick_chunk(h, h->n_rows(), T);
   const int n_chunks = (T + chunk - 1) / chunk;
-  const size_t slots = (size_t)h->B * h->cfg.n_heads * n_chunks;
+  const size_t slots = (size_t)h->n_rows() * h->cfg.n_heads * n_chunks;
   const size_t acc_bytes = align_up(slots * h->hd * sizeof(float)), ml_bytes = slots * 2 * sizeof(float);
   if (acc_bytes + ml_bytes > kStaticScratchBytes) return SD_ERR_CAPACITY;   // split-KV partials beyond the static array
   void* base = nullptr;
@@ -729,10 +782,10 @@ int sd_decode_step_host(sd_handle* h, const int32_t* h_ids, int position, float*
   if (!h->have_schedule || !h->have_prefill) return SD_ERR_STATE;
   int32_t* d_ids = h->at<int32_t>(h->A.ids);
   float* d_logits = h->at<float>(h->A.logits);
-  if (cudaMemcpyAsync(d_ids, h_ids, (size_t)h->B * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  if (cudaMemcpyAsync(d_ids, h_ids, (size_t)h->n_rows() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
   const int err = decode_step_impl(h, d_ids, position, d_logits);
   if (err) return err;
-  if (cudaMemcpyAsync(h_logits, d_logits, (size_t)h->B * h->cfg.vocab * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+  if (cudaMemcpyAsync(h_logits, d_logits, (size_t)h->n_rows() * h->cfg.vocab * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
       cudaStreamSynchronize(h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
   return SD_OK;
 }
