@@ -69,11 +69,11 @@ def step_bytes(wl: synth.Workload, n_active) -> float:
 # --------------------------------------------------------------------------- ncu traffic of the dominant kernel
 
 # DRAM bytes (read + write) per algorithmic byte of attn_partial_kernel, from an ncu --set full
-# capture at config 4's launch shape (1.08695 GB moved for 1.07583 GB of K and V at T = 1026; the
+# capture at config 4's launch shape (1.0825 GB moved for 1.07688 GB of K and V at T = 1027; the
 # traffic is proportional to T; a summary of the capture is kept under profiles/).  Valid only for the kernel source it was
 # taken on: the hash below is checked and `traffic` is null once the kernel text has changed.
-ATTN_TRAFFIC_RATIO = 1.0104
-ATTN_KERNEL_SHA256 = "1869cf8f40bc46c57d62cbbb198d42064b05ac355f561f429b98728d11566cd2"
+ATTN_TRAFFIC_RATIO = 1.0057
+ATTN_KERNEL_SHA256 = "31a94a145b5ed8ac87c0b55544c26e415ec060262f217260c54eeee81869bd3d"
 
 
 def attention_kernel_hash() -> str:
@@ -237,6 +237,8 @@ def gpu_arm(args, wl, rank, world):
         dec.set_option(binding.SD_OPT_GEMM, args.gemm_mode)
     if args.cluster:
         dec.set_option(binding.SD_OPT_CLUSTER, args.cluster)
+    if args.issuers:
+        dec.set_option(binding.SD_OPT_GEMM_ISSUERS, args.issuers)
     if args.pdl is not None:
         dec.set_option(binding.SD_OPT_PDL, args.pdl)
     if args.attn_chunk:
@@ -418,6 +420,7 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA graph replay (profiler runs)")
     ap.add_argument("--gemm-mode", type=int, default=0, help="SD_OPT_GEMM (0 automatic, 1 CUDA cores, 2 128-row kernel)")
     ap.add_argument("--cluster", type=int, default=0, help="SD_OPT_CLUSTER (0 automatic)")
+    ap.add_argument("--issuers", type=int, default=0, help="SD_OPT_GEMM_ISSUERS (1 or 2; 0 = library default)")
     ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")

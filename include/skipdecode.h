@@ -262,8 +262,10 @@ enum {
   SD_OPT_CLUSTER = 6,      /* blocks per cluster that split K in the cluster GEMMs: 0 = automatic, 1..4
                               (the token-stationary kernel uses 1 or 2)                               */
   SD_OPT_WEIGHT_TILES = 7, /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
-  SD_OPT_PREFILL_ATTN = 8  /* 1 (default): sd_prefill's causal attention runs as 64x64 tensor-core tiles
+  SD_OPT_PREFILL_ATTN = 8, /* 1 (default): sd_prefill's causal attention runs as 64x64 tensor-core tiles
                               (bf16 storage, head size 64 or 128); 0: one decode-style block per query row */
+  SD_OPT_GEMM_ISSUERS = 9  /* MMA-issuing warps per block of the 128-row GEMM at up to 64 tokens: 1 or 2
+                              (2: alternate k-blocks go to two accumulators that the epilogue adds)       */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff

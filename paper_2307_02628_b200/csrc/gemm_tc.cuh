@@ -141,14 +141,16 @@ __host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb
 __host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
 
-template <int NB, int EPI>
-__global__ void __launch_bounds__(192, 1)
+// ISS = 2: a second MMA-issuing warp (warp 6).  The two issuers take alternate k-blocks into
+// accumulators of their own (tensor-memory columns [0, 2 NB) and [2 NB, 4 NB)); the epilogue adds them.
+template <int NB, int EPI, int ISS = 1>
+__global__ void __launch_bounds__(192 + 32 * (ISS - 1), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                int kb_per_split, int* __restrict__ status, const QkvOut qo) {
   constexpr int STAGES = stages_for(NB);
   constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
-  constexpr int TMEM_COLS = 2 * NB;              // W.hi in columns [0, NB), W.lo in [NB, 2 NB): power of two >= 32
+  constexpr int TMEM_COLS = 2 * NB * ISS;        // per issuer: W.hi in columns [0, NB), W.lo in [NB, 2 NB); a power of two >= 32
   constexpr int CW = NB < 32 ? 16 : 32;          // accumulator columns read per tcgen05.ld
 
   extern __shared__ uint8_t smem_raw[];
@@ -169,7 +171,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    mbar_init(accum_bar, 1);
+    mbar_init(accum_bar, (ISS == 2 && nkb > 1) ? 2 : 1);        // one arrival per issuer that has k-blocks
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -218,15 +220,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || (ISS == 2 && warp == 6)) {
     if (lane == 0) {
+      const int w = warp == 1 ? 0 : 1;            // which issuer
       // The hi tile (NB rows) and the lo tile (NB rows) sit back to back in the stage, so they are
       // one K-major operand of 2 NB rows: a single MMA of N = 2 NB per k-step puts W.hi and W.lo
       // side by side in tensor memory (the epilogue adds the halves).  One wide instruction
       // instead of two narrow ones: at these sizes the MMA pipe is paced per instruction.
       constexpr uint32_t idesc = instr_desc(2 * NB);
       bool ok = true;
-      for (int i = 0; i < nkb && ok; ++i) {
+      for (int i = w; i < nkb && ok; i += ISS) {
         const int s = i % STAGES, round = i / STAGES;
         ok = mbar_wait(full0 + 8 * s, round & 1, abort_flag, status);
         if (!ok) break;
@@ -235,10 +238,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const uint64_t a_desc = smem_desc(a_addr), b_desc = smem_desc(a_addr + A_BYTES);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k)     // 32 bytes further along K inside the swizzle row
-          umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          umma(tmem_base + (uint32_t)(w * 2 * NB), a_desc + 2 * k, b_desc + 2 * k, idesc, (i > w || k > 0) ? 1u : 0u);
         umma_commit(empty0 + 8 * s);              // the stage is free once these MMAs have read it
       }
-      if (ok) umma_commit(accum_bar);             // accumulator complete
+      if (ok && (w == 0 || nkb > 1)) umma_commit(accum_bar);   // this issuer's accumulator is complete
     }
   } else {
     pdl_wait();                                   // bias aside, the epilogue reads and writes buffers earlier kernels own
@@ -277,6 +280,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
         if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (ISS == 2 && nkb > 1) {                // the second issuer's partial sums
+          uint32_t r2[32], rl2[32];
+          if (CW == 32) { tmem_ld32(taddr + 2 * NB, r2); tmem_ld32(taddr + 3 * NB, rl2); } else { tmem_ld16(taddr + 2 * NB, r2); tmem_ld16(taddr + 3 * NB, rl2); }
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < CW; ++j) {
+            r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+            rl[j] = __float_as_uint(__uint_as_float(rl[j]) + __uint_as_float(rl2[j]));
+          }
+        }
         if (n < N) {
 #pragma unroll
           for (int j = 0; j < CW; ++j) {
@@ -336,13 +349,17 @@ struct TcContext {
   int ready = 0;
   int sm_count = 148;
   bool pdl = false;      // launch with the programmatic-dependent-launch attribute
+  int issuers = 1;       // MMA-issuing warps per block (2 only for token tiles of at most 64)
   // (pointer, rows, cols, box rows) -> tensor map of a row-major bf16 matrix, 64-column boxes, 128-byte swizzle
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
 };
 
 template <int NB, int EPI>
 inline bool tc_prepare() {
-  return cudaFuncSetAttribute(tc::gemm_tc_kernel<NB, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(NB)) == cudaSuccess;
+  if (NB <= 64 &&
+      cudaFuncSetAttribute(tc::gemm_tc_kernel<NB, EPI, (NB <= 64 ? 2 : 1)>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(NB)) != cudaSuccess)
+    return false;
+  return cudaFuncSetAttribute(tc::gemm_tc_kernel<NB, EPI, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(NB)) == cudaSuccess;
 }
 template <int NB>
 inline bool tc_prepare_nb() {
@@ -390,19 +407,20 @@ inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int co
   return &c.maps.emplace(key, m).first->second;
 }
 
-template <int NB>
+template <int NB, int ISS>
 inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
                       int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status, const tc::QkvOut& qo) {
   dim3 grid((N + tc::BM - 1) / tc::BM, (M + NB - 1) / NB, splits);
+  const dim3 block(192 + 32 * (ISS - 1));
   const int smem = tc::smem_bytes(NB);
   if (epi == EPI_STORE_F32)
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_STORE_F32>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_STORE_F32, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else if (epi == EPI_RELU_T)
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RELU_T>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RELU_T, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else if (epi == EPI_QKV_CACHE)
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_QKV_CACHE>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_QKV_CACHE, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32>, grid, dim3(192), smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   return true;
 }
 
@@ -428,11 +446,18 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   }
   int kb_per_split = (kb_total + splits - 1) / splits;
   splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split
+  if (c.issuers == 2 && nb <= 64) {
+    switch (nb) {
+      case 16: return tc_launch<16, 2>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+      case 32: return tc_launch<32, 2>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+      default: return tc_launch<64, 2>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    }
+  }
   switch (nb) {
-    case 16: return tc_launch<16>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    case 32: return tc_launch<32>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    case 64: return tc_launch<64>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    default: return tc_launch<128>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 16: return tc_launch<16, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 32: return tc_launch<32, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 64: return tc_launch<64, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    default: return tc_launch<128, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
   }
 }
 template <typename T>

@@ -839,6 +839,10 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value < 0 || value > sd::tcw::MAX_CLUSTER) return SD_ERR_ARG;
       if (value != h->wide.force_cluster) drop_graphs(h);
       h->wide.force_cluster = value; return SD_OK;
+    case SD_OPT_GEMM_ISSUERS:
+      if (value != 1 && value != 2) return SD_ERR_ARG;
+      if (value != h->tc.issuers) drop_graphs(h);
+      h->tc.issuers = value; return SD_OK;
     case SD_OPT_PREFILL_ATTN:
       h->opt_prefill = value ? 1 : 0; return SD_OK;
     case SD_OPT_WEIGHT_TILES:
