@@ -148,7 +148,11 @@ __global__ void __launch_bounds__(192 + 32 * (ISS - 1), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                int kb_per_split, int* __restrict__ status, const QkvOut qo) {
-  constexpr int STAGES = stages_for(NB);
+  // With two issuers the stage count is even, so that a stage always belongs to the same issuer (k-block
+  // i, stage i % STAGES and issuer i & 1 then agree in parity).  A phase-parity wait is only safe for a
+  // thread that has itself consumed the stage's previous round: another thread, one round ahead of a
+  // slower consumer, would take the barrier's still-incomplete phase for the one before it.
+  constexpr int STAGES = ISS == 2 ? (stages_for(NB) & ~1) : stages_for(NB);
   constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
   constexpr int TMEM_COLS = 2 * NB * ISS;        // per issuer: W.hi in columns [0, NB), W.lo in [NB, 2 NB); a power of two >= 32
   constexpr int CW = NB < 32 ? 16 : 32;          // accumulator columns read per tcgen05.ld
