@@ -205,7 +205,8 @@ class Decoder:
     def decode_step(self, ids: torch.Tensor, position: int, logits: torch.Tensor | None = None) -> torch.Tensor:
         ids = self._dev_i32(ids)
         n = getattr(self, "_n_rows", None) or self.B
-        assert ids.numel() == n, f"{ids.numel()} token ids for {n} generating rows"
+        if n is not None:              # before a prefill the library itself reports the state error
+            assert ids.numel() == n, f"{ids.numel()} token ids for {n} generating rows"
         if logits is None:
             logits = torch.empty(ids.shape[0], self.shape.vocab, dtype=torch.float32, device=self.device)
         self._order()

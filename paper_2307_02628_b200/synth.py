@@ -75,6 +75,18 @@ CONFIGS = {
 }
 
 
+# Table 2's presets (base layers -> {target speed-up: (warm-up, min, max)}) at the sequence envelopes of
+# the paper's three datasets (Section 3.2: prompt / total length 60/160, 512/1024, 1024/2048), batch 64:
+# "t2-6.7b-3x-reddit" and so on.  Same synthetic tokens and weights as the five configurations above.
+TABLE2 = {"6.7b": (OPT_6B7, {2: (1, 11, 22), 3: (1, 8, 14), 4: (1, 6, 10), 5: (1, 5, 8)}),
+          "1.3b": (OPT_1B3, {2: (1, 8, 16), 3: (1, 6, 10), 4: (1, 5, 7), 5: (1, 4, 6)})}
+ENVELOPES = {"e2e": (60, 100), "reddit": (512, 512), "cnndm": (1024, 1024)}
+for _model, (_shape, _rows) in TABLE2.items():
+    for _k, (_w, _mn, _mx) in _rows.items():
+        for _ds, (_p, _g) in ENVELOPES.items():
+            CONFIGS[f"t2-{_model}-{_k}x-{_ds}"] = Workload(_shape, 64, _p, _g, _mx, _mn, _w)
+
+
 def _seed_for(seed: int, name: str) -> int:
     h = hashlib.sha256(f"{seed}:{name}".encode()).digest()
     return int.from_bytes(h[:8], "little") & 0x7FFFFFFFFFFFFFFF

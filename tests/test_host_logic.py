@@ -37,6 +37,30 @@ def test_schedule_rejects_bad_arguments(args):
     assert e.value.code == binding.SD_ERR_ARG
 
 
+def test_table2_presets_are_the_papers_rows():
+    # every preset workload carries the (warm-up, min, max) of its row of Table 2 and the schedule's mean
+    # layer count is the row's midpoint, the figure the target speed-up is computed from
+    import os
+    rows = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "table2_budgets.txt")):
+        if line.strip() and not line.startswith("#"):
+            base, speed, avg, warm, mn, mx = line.split()
+            rows[(int(base), int(speed))] = (int(warm), int(mn), int(mx))
+    assert len(rows) == 8
+    seen = 0
+    for name, wl in synth.CONFIGS.items():
+        if not name.startswith("t2-"):
+            continue
+        _, model, speed, ds = name.split("-")
+        assert (wl.warmup, wl.min_layers, wl.max_layers) == rows[(wl.shape.n_layers, int(speed[0]))]
+        assert (wl.prompt_len, wl.gen_len) == synth.ENVELOPES[ds] and wl.prompt_len + wl.gen_len <= wl.shape.max_pos
+        n, top = binding.schedule_compute(wl.shape.n_layers, wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len)
+        assert abs(sum(n) / len(n) - (wl.max_layers + wl.min_layers) / 2) <= 0.5 / len(n) + 1e-9 or wl.gen_len % 2 == 0
+        assert n[0] == wl.max_layers and n[-1] == wl.min_layers
+        seen += 1
+    assert seen == 24
+
+
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4", "c5"])
 def test_cache_plan_matches_the_active_sets(name):
     wl = synth.CONFIGS[name]
