@@ -202,7 +202,8 @@ def bench_config(wl, args):
     return {"workload": f"{args.config}: {s.name} L{s.n_layers} d{s.d_model} H{s.n_heads} f{s.d_ffn} V{s.vocab} {s.dtype}, "
                         f"batch {wl.batch}, prompt {wl.prompt_len}, gen {wl.gen_len}, linear budget {wl.max_layers}->{wl.min_layers} top layers, warm-up {wl.warmup}",
             "global_batch": wl.batch * args.gpus, "l2": "inputs larger than L2 (KV cache and weights are GBs)",
-            "tokens": "greedy on device (value); forced ids from host (e2e)"}
+            "tokens": ("greedy on device" if args.select == "greedy" else "top-p 0.7, temperature 0.3 on device, seeded uniforms")
+                      + " (value); forced ids from host (e2e)"}
 
 
 # --------------------------------------------------------------------------- GPU arm
@@ -258,13 +259,24 @@ def gpu_arm(args, wl, rank, world):
 
     G_run = G if args.max_gen_steps <= 0 else min(G, args.max_gen_steps)   # < G only for profiler runs
 
+    # the paper's own token selection (Section 3.2) instead of greedy: one seeded uniform per (step, row)
+    uniforms = None
+    if args.select == "top-p":
+        uniforms = torch.stack([synth.make_uniforms(B, seed=1000 + g) for g in range(G + 1)]).to(device)
+
+    def choose(d, lg, g):
+        if uniforms is None:
+            d.greedy(lg, ids)
+        else:
+            d.sample_top_p(lg, uniforms[g], 0.3, 0.7, ids)
+
     def one_pass(nsteps=None, d=None):
         d = d or dec
         d.rewind()
-        d.greedy(logits0, ids)
+        choose(d, logits0, 0)
         for g in range(G_run if nsteps is None else nsteps):
             d.decode_step(ids, P + g, logits)
-            d.greedy(logits, ids)
+            choose(d, logits, g + 1)
 
     def timed(fn, reps):
         barrier()
@@ -420,6 +432,8 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA graph replay (profiler runs)")
     ap.add_argument("--gemm-mode", type=int, default=0, help="SD_OPT_GEMM (0 automatic, 1 CUDA cores, 2 128-row kernel)")
     ap.add_argument("--cluster", type=int, default=0, help="SD_OPT_CLUSTER (0 automatic)")
+    ap.add_argument("--select", default="greedy", choices=["greedy", "top-p"],
+                    help="token selection in the timed generation loop (the five configurations are greedy)")
     ap.add_argument("--issuers", type=int, default=0, help="SD_OPT_GEMM_ISSUERS (1 or 2; 0 = library default)")
     ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
