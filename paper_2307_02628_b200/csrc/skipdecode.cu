@@ -802,8 +802,20 @@ int sd_sample_top_p(sd_handle* h, const float* d_logits, int B, float temperatur
   if (!h || !d_logits || !d_uniforms || !d_next || B < 1) return SD_ERR_ARG;
   if (!std::isfinite(temperature) || !(temperature > 0.0f) || !std::isfinite(top_p) || !(top_p > 0.0f) || top_p > 1.0f)
     return SD_ERR_ARG;
-  sd::sample_top_p_kernel<<<B, sd::SAMPLE_THREADS, 0, h->stream>>>(d_logits, h->cfg.vocab, d_uniforms,
-                                                                  1.0f / temperature, top_p, d_next);
+  const int vocab = h->cfg.vocab;
+  if (vocab <= sd::SAMPLE_MAX_SMEM_VOCAB) {        // the row is staged in shared memory
+    static bool configured = false;
+    if (!configured) {
+      if (cudaFuncSetAttribute(sd::sample_top_p_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               sd::SAMPLE_MAX_SMEM_VOCAB * 4) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+      configured = true;
+    }
+    sd::sample_top_p_kernel<true><<<B, sd::SAMPLE_THREADS, (size_t)vocab * 4, h->stream>>>(d_logits, vocab, d_uniforms,
+                                                                                        1.0f / temperature, top_p, d_next);
+  } else {
+    sd::sample_top_p_kernel<false><<<B, sd::SAMPLE_THREADS, 0, h->stream>>>(d_logits, vocab, d_uniforms,
+                                                                           1.0f / temperature, top_p, d_next);
+  }
   h->launches += 1;
   return cudaGetLastError() == cudaSuccess ? SD_OK : SD_ERR_CUDA;
 }
