@@ -264,8 +264,11 @@ enum {
   SD_OPT_WEIGHT_TILES = 7, /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
   SD_OPT_PREFILL_ATTN = 8, /* 1 (default): sd_prefill's causal attention runs as 64x64 tensor-core tiles
                               (bf16 storage, head size 64 or 128); 0: one decode-style block per query row */
-  SD_OPT_GEMM_ISSUERS = 9  /* MMA-issuing warps per block of the 128-row GEMM at up to 64 tokens: 1 or 2
+  SD_OPT_GEMM_ISSUERS = 9, /* MMA-issuing warps per block of the 128-row GEMM at up to 64 tokens: 1 or 2
                               (2: alternate k-blocks go to two accumulators that the epilogue adds)       */
+  SD_OPT_GEMM_PERSISTENT = 10 /* 1 (default): products with more than 64 tokens and more output tiles than SMs
+                              run on the persistent kernel (one block per SM, double-buffered accumulator,
+                              epilogue overlapped with the next tile's main loop); 0: one block per tile */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff

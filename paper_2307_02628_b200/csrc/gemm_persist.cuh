@@ -1,0 +1,258 @@
+// Persistent variant of the 128-row tensor-core GEMM for token tiles of 128 (prompt pass, batches
+// above 64): one CTA per SM walks over many output tiles, and the accumulator is double-buffered in
+// tensor memory (2 x 256 columns), so the epilogue of tile i (TMEM -> registers -> global) runs
+// while the MMA warp is already issuing tile i + 1 and the producer keeps the shared-memory ring
+// full across tile boundaries.  Same operands, tile shapes, descriptors and epilogues as
+// gemm_tc_kernel<128, EPI>; no split-K (there are at least as many tiles as SMs where it is used).
+//
+// Barriers: full[s] / empty[s] per pipeline stage as in the one-tile kernel, plus per accumulator
+// buffer tfull[b] (MMA warp -> epilogue: accumulator complete) and tempty[b] (128 epilogue threads ->
+// MMA warp: accumulator read out).  Every wait is bounded and reports through the status word.
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace sd {
+
+namespace tcp {
+using namespace tc;
+
+constexpr int NB = 128;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
+constexpr int ACC_COLS = 2 * NB;                 // one accumulator: W.hi in [0, NB), W.lo in [NB, 2 NB)
+constexpr int TMEM_COLS = 2 * ACC_COLS;          // two accumulators = all 512 columns
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/;
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                       const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
+                       int tiles_n, int tiles_total, int* __restrict__ status, const QkvOut qo) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  uint8_t* tiles_ptr = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES);
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * STAGES, tfull0 = full0 + 16 * STAGES, tempty0 = tfull0 + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  long long* col_row = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [NB], QKV epilogue only
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nkb = K / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+      // the first stages' weight tiles depend on nothing: stream them before waiting for the previous kernel
+      const int first_tile = blockIdx.x;
+      const int early = nkb < STAGES ? nkb : STAGES;
+      {
+        const int n0 = (first_tile % tiles_n) * BM;
+        for (int i = 0; i < early; ++i) {
+          const uint32_t fb = full0 + 8 * i;
+          mbar_expect_tx(fb, STAGE_BYTES);
+          load_w_tile(tiles + i * STAGE_BYTES, &map_w, qo, i, n0, fb);
+        }
+      }
+      pdl_wait();
+      int it = 0;
+      bool ok = true;
+      for (int tile = first_tile; tile < tiles_total && ok; tile += gridDim.x) {
+        const int n0 = (tile % tiles_n) * BM, m0 = (tile / tiles_n) * NB;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % STAGES, round = it / STAGES;
+          const uint32_t fb = full0 + 8 * s;
+          const uint32_t a_dst = tiles + s * STAGE_BYTES;
+          if (it >= early) {
+            if (round > 0 && !mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) { ok = false; break; }
+            mbar_expect_tx(fb, STAGE_BYTES);
+            load_w_tile(a_dst, &map_w, qo, kb, n0, fb);
+          }
+          tma_load_2d(a_dst + A_BYTES, &map_x, kb * BK, m0, fb);                 // hi part: columns [0, K)
+          tma_load_2d(a_dst + A_BYTES + B_BYTES, &map_x, K + kb * BK, m0, fb);   // lo part: columns [K, 2K)
+        }
+      }
+      if (*abort_flag) {
+        // drain: wait (bounded) until every copy issued has landed before the CTA exits
+        const int issued = it > early ? it : early;
+        const int first = issued > STAGES ? issued - STAGES : 0;
+        for (int i = first; i < issued; ++i) {
+          const long long t0 = clock64();
+          while (!mbar_try(full0 + 8 * (i % STAGES), (i / STAGES) & 1) && clock64() - t0 < kWaitLimit) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(2 * NB);
+      int it = 0, i = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < tiles_total && ok; tile += gridDim.x, ++i) {
+        const int buf = i & 1, use = i >> 1;
+        if (use > 0) ok = mbar_wait(tempty0 + 8 * buf, (use - 1) & 1, abort_flag, status);   // the epilogue has read this accumulator out
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = tmem_base + (uint32_t)(buf * ACC_COLS);
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % STAGES, round = it / STAGES;
+          ok = mbar_wait(full0 + 8 * s, round & 1, abort_flag, status);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = tiles + s * STAGE_BYTES;
+          const uint64_t a_desc = smem_desc(a_addr), b_desc = smem_desc(a_addr + A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(empty0 + 8 * s);
+        }
+        if (ok) umma_commit(tfull0 + 8 * buf);
+      }
+    }
+  } else {
+    pdl_wait();
+    const int quarter = warp & 3;
+    const int t_epi = threadIdx.x - 64;           // 0..127 over the four epilogue warps
+    int i = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < tiles_total && ok; tile += gridDim.x, ++i) {
+      const int buf = i & 1, use = i >> 1;
+      const int n0 = (tile % tiles_n) * BM, m0 = (tile / tiles_n) * NB;
+      const int n = n0 + quarter * 32 + lane;
+      int kv_head = 0, kv_elem = 0;
+      __nv_bfloat16* kv_base = nullptr;
+      if (EPI == EPI_QKV_CACHE) {
+        int b, pos;
+        qo.map.get(m0 + t_epi, b, pos);
+        col_row[t_epi] = (m0 + t_epi < M && pos < qo.cap) ? (long long)b * qo.H * qo.cap + pos : -1;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (n >= qo.d && n < N) {
+          const int cc = n < 2 * qo.d ? n - qo.d : n - 2 * qo.d;
+          kv_head = cc / qo.hd;
+          kv_elem = cc - kv_head * qo.hd;
+          kv_base = n < 2 * qo.d ? qo.Kc : qo.Vc;
+        }
+      }
+      ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, status);
+      if (tile + (int)gridDim.x >= tiles_total) pdl_launch_dependents();   // this CTA's last main loop is over
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const float b = (bias != nullptr && n < N) ? __bfloat162float(bias[n]) : 0.f;
+#pragma unroll 1
+      for (int c = 0; c < NB; c += 32) {
+        uint32_t r[32], rl[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * ACC_COLS + c);
+        tmem_ld32(taddr, r);
+        tmem_ld32(taddr + NB, rl);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (n < N) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int m = m0 + c + j;
+            if (m < M) {
+              const float v = (__uint_as_float(r[j]) + __uint_as_float(rl[j])) + b;
+              const size_t idx = (size_t)m * ldo + n;
+              if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
+              else if (EPI == EPI_QKV_CACHE) {
+                if (kv_base == nullptr) {
+                  reinterpret_cast<float*>(out)[idx] = v;
+                } else {
+                  const long long row = col_row[c + j];
+                  if (row >= 0) kv_base[((size_t)row + (size_t)kv_head * qo.cap) * qo.hd + kv_elem] = __float2bfloat16_rn(v);
+                }
+              }
+              else if (EPI == EPI_RELU_T)
+                Operand<__nv_bfloat16>::store(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)m * ldo, N, n, fmaxf(v, 0.f));
+              else atomicAdd(reinterpret_cast<float*>(out) + idx, v);
+            }
+          }
+        }
+      }
+      // this thread's reads of the accumulator are complete: hand the buffer back to the MMA warp
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(tempty0 + 8 * buf);
+      if (EPI == EPI_QKV_CACHE) asm volatile("bar.sync 1, 128;" ::: "memory");   // col_row is rewritten for the next tile
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace tcp
+
+struct PersistContext { int ready = 0; int enabled = 1; };
+
+template <int EPI>
+inline bool persist_prepare() {
+  return cudaFuncSetAttribute(tcp::gemm_tc_persist_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tcp::SMEM_BYTES) == cudaSuccess;
+}
+inline void persist_init(PersistContext& p, const TcContext& c) {
+  if (!c.ready) return;
+  if (!(persist_prepare<EPI_STORE_F32>() && persist_prepare<EPI_RELU_T>() && persist_prepare<EPI_RESIDUAL_F32>() &&
+        persist_prepare<EPI_QKV_CACHE>())) {
+    cudaGetLastError();
+    return;
+  }
+  p.ready = 1;
+}
+
+// Takes the product when the token tile is 128 and there are more tiles than SMs (so that K is not split);
+// false leaves it to tc_gemm.
+inline bool persist_gemm(PersistContext& p, TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const __nv_bfloat16* W,
+                         const __nv_bfloat16* bias, int M, int N, int K, void* out, int ldo, int epi, int* status,
+                         const tc::QkvOut* qkv_out = nullptr, const __nv_bfloat16* Wp = nullptr) {
+  if (!p.ready || !p.enabled || !c.ready || K % tc::BK || M <= 64 || N < 1) return false;
+  if (epi == EPI_QKV_CACHE && (!qkv_out || qkv_out->d % tc::BM || N != 3 * qkv_out->d)) return false;
+  if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
+  const int tiles_n = (N + tc::BM - 1) / tc::BM, tiles_m = (M + tcp::NB - 1) / tcp::NB;
+  const int total = tiles_n * tiles_m;
+  if (total <= c.sm_count) return false;
+  if (K / tc::BK > 128) return false;       // long main loops hide little behind them (measured: fc2 3 % slower here)
+  tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
+  qo.packed_kb = Wp ? K / tc::BK : 0;
+  qo.w_packed = Wp;
+  const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
+  const CUtensorMap* mx = tc_map(c, X, M, 2 * K, tcp::NB);
+  if (!mw || !mx) return false;
+  const dim3 grid(c.sm_count), block(192);
+  if (epi == EPI_STORE_F32)
+    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_STORE_F32>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  else if (epi == EPI_RELU_T)
+    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_RELU_T>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  else if (epi == EPI_QKV_CACHE)
+    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_QKV_CACHE>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  else
+    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_RESIDUAL_F32>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  return true;
+}
+template <typename T>
+inline bool persist_gemm(PersistContext&, TcContext&, cudaStream_t, const T*, const T*, const T*, int, int, int, void*, int, int, int*,
+                         const tc::QkvOut* = nullptr, const T* = nullptr) {
+  return false;
+}
+
+}  // namespace sd

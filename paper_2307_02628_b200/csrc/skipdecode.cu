@@ -17,6 +17,7 @@
 #include "gemm_tc.cuh"
 #include "gemm_wide.cuh"
 #include "gemm_xs.cuh"
+#include "gemm_persist.cuh"
 #include "sample.cuh"
 #include "attn_prefill.cuh"
 
@@ -79,6 +80,7 @@ struct sd_handle {
   sd::TcContext tc;
   sd::WideContext wide;
   sd::XsContext xs;
+  sd::PersistContext persist;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(arena + off); }
   int* status() const { return at<int>(A.scalars); }
@@ -185,7 +187,9 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   A.logits = take((size_t)c.max_batch * c.vocab * 4);
   A.scalars = take(256);
   A.pad = take((size_t)c.max_batch * 4);     // left-padding slots per batch row (ragged prompts)
-  A.rows = take((size_t)c.max_batch * 4);    // batch rows still generating
+  // batch rows still generating; a GEMM epilogue looks up whole token tiles (up to 127 entries past the
+  // row count, results unused), so the array is that much longer than the batch
+  A.rows = take(((size_t)c.max_batch + 128) * 4);
   A.total = off;
 }
 
@@ -238,6 +242,7 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_of
   if (std::is_same<T, bf16>::value && h->opt_gemm != 1) {
     if (h->opt_gemm == 4) done = sd::xs_gemm(h->xs, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp, h->wide.force_cluster);
     if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
+    if (!done) done = sd::persist_gemm(h->persist, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
     if (!done) done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
   }
   if (!done) {
@@ -269,6 +274,7 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
   bool done = false;
   if (h->opt_gemm == 4) done = sd::xs_gemm(h->xs, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp, h->wide.force_cluster);
   if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
+  if (!done) done = sd::persist_gemm(h->persist, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (done) Lc.end(); else Lc.cancel();
   return done;
@@ -572,6 +578,7 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
   sd::tc_init(h->tc);
   sd::wide_init(h->wide, h->tc);
   sd::xs_init(h->xs, h->tc);
+  sd::persist_init(h->persist, h->tc);
   if (h->tc.ready && h->A.packable) {            // tile-packed copies of the matrices, made once
     const int d = cfg->d_model, f = cfg->d_ffn;
     auto pack = [&](const void* W, size_t off, int n, int k) {
@@ -855,6 +862,9 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != 1 && value != 2) return SD_ERR_ARG;
       if (value != h->tc.issuers) drop_graphs(h);
       h->tc.issuers = value; return SD_OK;
+    case SD_OPT_GEMM_PERSISTENT:
+      if ((value != 0) != (h->persist.enabled != 0)) drop_graphs(h);
+      h->persist.enabled = value ? 1 : 0; return SD_OK;
     case SD_OPT_PREFILL_ATTN:
       h->opt_prefill = value ? 1 : 0; return SD_OK;
     case SD_OPT_WEIGHT_TILES:

@@ -308,6 +308,29 @@ def test_one_and_two_mma_issuers_agree(B):
     assert float((runs[1] - runs[2]).abs().max()) <= 1e-3
 
 
+@pytest.mark.parametrize("B,P", [(32, 128), (40, 100)])
+def test_persistent_gemm_in_the_prompt_pass(B, P):
+    # enough 128-token tiles per product (more than SMs) for the persistent kernel to take the QKV, out-proj,
+    # fc1 and fc2 products of the prompt pass; the second case ends in a partial token tile
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("persist-bf16", 2, 768, 6, 1024, 640, 160, "bf16")
+    wl = synth.Workload(shape, B, P, 4, 2, 1, 0)
+    w = synth.make_weights(shape, seed=14, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    rows = synth.sample_rows(B, 6)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced, rows=rows)
+    runs = {}
+    for persistent in (1, 0):
+        dec = harness.make_decoder(wl, w)
+        dec.set_option(binding.SD_OPT_GEMM_PERSISTENT, persistent)
+        runs[persistent] = harness.gpu_run_forced(dec, wl, prompts, forced, rows=rows)
+        dec.close()
+        err, strict, near = harness.compare(runs[persistent], ref, harness.TOL["bf16"])
+        print(f"persistent={persistent} B={B} P={P}: max|err|={err:.3e} argmax strict={strict:.4f} near={near:.4f}")
+        assert err <= harness.TOL["bf16"] and near >= 0.99
+    assert float((runs[1] - runs[0]).abs().max()) <= 2e-3     # same products; the residual adds arrive in another order
+
+
 @pytest.mark.parametrize("alpha", [2, 3])
 def test_power_law_budget_table(alpha):
     """A caller-supplied budget table (power-law decay with warm-up 1) through sd_schedule_custom."""
