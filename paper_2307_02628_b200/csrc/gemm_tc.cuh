@@ -137,6 +137,11 @@ __device__ __forceinline__ void load_w_tile(uint32_t dst, const CUtensorMap* map
     tma_load_2d(dst, map, kb * BK, n_row0, bar);
 }
 
+// Epilogue warps: a warp can only read the quarter of the tensor-memory lanes that matches its index
+// mod 4, so there are four warps per group; with two groups each takes half of the token columns,
+// which halves the serial part of the epilogue (loads from tensor memory, then one store per column).
+__host__ __device__ constexpr int epi_warps(int nb) { return nb >= 32 ? 8 : 4; }
+__host__ __device__ constexpr int block_threads(int nb, int iss) { return 64 + 32 * epi_warps(nb) + 32 * (iss - 1); }
 __host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
 __host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
@@ -144,7 +149,7 @@ __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * s
 // ISS = 2: a second MMA-issuing warp (warp 6).  The two issuers take alternate k-blocks into
 // accumulators of their own (tensor-memory columns [0, 2 NB) and [2 NB, 4 NB)); the epilogue adds them.
 template <int NB, int EPI, int ISS = 1>
-__global__ void __launch_bounds__(192 + 32 * (ISS - 1), 1)
+__global__ void __launch_bounds__(block_threads(NB, ISS), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                int kb_per_split, int* __restrict__ status, const QkvOut qo) {
@@ -155,7 +160,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   constexpr int STAGES = ISS == 2 ? (stages_for(NB) & ~1) : stages_for(NB);
   constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
   constexpr int TMEM_COLS = 2 * NB * ISS;        // per issuer: W.hi in columns [0, NB), W.lo in [NB, 2 NB); a power of two >= 32
-  constexpr int CW = NB < 32 ? 16 : 32;          // accumulator columns read per tcgen05.ld
+  constexpr int EW = epi_warps(NB);              // epilogue warps: 4, or 8 = two groups that split the columns
+  constexpr int GROUP_COLS = NB / (EW / 4);      // token columns per group of four warps
+  constexpr int CW = GROUP_COLS < 32 ? 16 : 32;  // accumulator columns read per tcgen05.ld
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -224,7 +231,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
       }
     }
-  } else if (warp == 1 || (ISS == 2 && warp == 6)) {
+  } else if (warp == 1 || (ISS == 2 && warp == 2 + EW)) {
     if (lane == 0) {
       const int w = warp == 1 ? 0 : 1;            // which issuer
       // The hi tile (NB rows) and the lo tile (NB rows) sit back to back in the stage, so they are
@@ -256,13 +263,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     int kv_head = 0, kv_elem = 0;
     __nv_bfloat16* kv_base = nullptr;
     if (EPI == EPI_QKV_CACHE) {
-      const int t = threadIdx.x - 64;             // 0..127 over the four epilogue warps
+      const int t = threadIdx.x - 64;             // 0.. over the epilogue warps
       if (t < NB) {
         int b, pos;
         qo.map.get(m0 + t, b, pos);
         col_row[t] = (m0 + t < M && pos < qo.cap) ? (long long)b * qo.H * qo.cap + pos : -1;
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * EW) : "memory");
       if (n >= qo.d && n < N) {
         const int cc = n < 2 * qo.d ? n - qo.d : n - 2 * qo.d;
         kv_head = cc / qo.hd;
@@ -279,7 +286,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const float b = (bias != nullptr && n < N && (EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
 #pragma unroll 1
-      for (int c = 0; c < NB; c += CW) {
+      const int c_begin = ((warp - 2) >> 2) * GROUP_COLS;
+      for (int c = c_begin; c < c_begin + GROUP_COLS; c += CW) {
         uint32_t r[32], rl[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
         if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
@@ -415,7 +423,7 @@ template <int NB, int ISS>
 inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
                       int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status, const tc::QkvOut& qo) {
   dim3 grid((N + tc::BM - 1) / tc::BM, (M + NB - 1) / NB, splits);
-  const dim3 block(192 + 32 * (ISS - 1));
+  const dim3 block(tc::block_threads(NB, ISS));
   const int smem = tc::smem_bytes(NB);
   if (epi == EPI_STORE_F32)
     launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_STORE_F32, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
