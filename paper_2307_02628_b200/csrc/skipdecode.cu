@@ -63,6 +63,7 @@ struct sd_handle {
   // ragged batches: left padding per row (host copy; device copy in the arena) and the rows still generating
   std::vector<int> pad, rows;
   bool have_pad = false, have_rows = false;
+  bool prefill_attn_ready = false, sample_ready = false;   // large dynamic shared memory enabled for these kernels
   int n_rows() const { return have_rows ? (int)rows.size() : B; }
   const int* d_pad() const { return have_pad ? at<int>(A.pad) : nullptr; }
   const int* d_rows() const { return have_rows ? at<int>(A.rows) : nullptr; }
@@ -306,13 +307,12 @@ template <int HD>
 bool launch_attention_prefill_hd(Launcher& Lc, const bf16* Kc, const bf16* Vc, int cap, int n_seq, int P, int b0) {
   sd_handle* h = Lc.h;
   constexpr int smem = 2 * 2 * sd::PF_BN * HD * 2;
-  static bool configured = false;
-  if (!configured) {
+  if (!h->prefill_attn_ready) {              // per handle: the attribute belongs to the handle's device
     if (cudaFuncSetAttribute(sd::attn_prefill_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
       cudaGetLastError();
       return false;
     }
-    configured = true;
+    h->prefill_attn_ready = true;
   }
   Lc.begin(SD_K_ATTENTION);
   dim3 grid((P + sd::PF_BM - 1) / sd::PF_BM, n_seq * h->cfg.n_heads);
@@ -811,11 +811,10 @@ int sd_sample_top_p(sd_handle* h, const float* d_logits, int B, float temperatur
     return SD_ERR_ARG;
   const int vocab = h->cfg.vocab;
   if (vocab <= sd::SAMPLE_MAX_SMEM_VOCAB) {        // the row is staged in shared memory
-    static bool configured = false;
-    if (!configured) {
+    if (!h->sample_ready) {                  // per handle: the attribute belongs to the handle's device
       if (cudaFuncSetAttribute(sd::sample_top_p_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                sd::SAMPLE_MAX_SMEM_VOCAB * 4) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
-      configured = true;
+      h->sample_ready = true;
     }
     sd::sample_top_p_kernel<true><<<B, sd::SAMPLE_THREADS, (size_t)vocab * 4, h->stream>>>(d_logits, vocab, d_uniforms,
                                                                                         1.0f / temperature, top_p, d_next);
