@@ -106,3 +106,15 @@ def test_sampling_small_vocabulary_and_generation():
         lr = ref.decode_step(ids_ref, wl.prompt_len + g)
     dec.close()
     assert agree >= 0.99 * wl.batch * wl.gen_len, agree
+
+
+def test_sampling_vocabulary_too_large_for_shared_memory():
+    # above 52 224 entries the row is not staged in shared memory and every pass reads it from global memory
+    shape = synth.ModelShape("toy-big-vocab", 1, 64, 1, 128, 60001, 16, "bf16")
+    wl = synth.Workload(shape, 6, 4, 2, 1, 1, 0)
+    dec = harness.make_decoder(wl, synth.make_weights(shape, seed=1))
+    for scale, step, temperature, top_p in ((1.0, 0.0, 0.3, 0.7), (2.0, 0.5, 1.0, 0.95), (0.2, 0.0, 0.3, 1.0)):
+        logits = synth.make_logits(6, shape.vocab, seed=31, scale=scale, step=step)
+        same, n = _compare(dec, logits, synth.make_uniforms(6, seed=32), temperature, top_p)
+        assert same == n
+    dec.close()
