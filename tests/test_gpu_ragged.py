@@ -103,3 +103,30 @@ def test_padding_content_is_invisible_and_errors():
         with pytest.raises(binding.SdError):
             dec.decode_step(torch.tensor([9, 5], dtype=torch.int32), 41)   # padding changed: prefill first
     dec.close()
+
+
+def test_host_buffer_and_static_scratch_steps_follow_the_row_list():
+    # the other two step entry points take and return exactly the generating rows as well
+    shape = synth.ModelShape("toy-ragged-64", 3, 256, 4, 384, 777, 160, "bf16")
+    wl = synth.Workload(shape, 5, 40, 4, 3, 2, 0)
+    w = synth.make_weights(shape, seed=12)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    rows = [1, 3, 4]
+    dec = harness.make_decoder(wl, w)
+    with torch.cuda.stream(dec.stream):
+        dec.schedule(3, 2, 0, 4)
+        dec.set_padding([0, 7, 0, 39, 12])
+        dec.prefill(prompts)
+        dec.set_rows(rows)
+        ids = forced[rows, 0].contiguous()
+        regular = dec.decode_step(ids, 40).cpu()
+        dec.rewind()
+        static = dec.decode_step_static(ids.to(dec.device), 40).cpu()
+        dec.rewind()
+        host = torch.empty(len(rows), shape.vocab, dtype=torch.float32).pin_memory()
+        dec.decode_step_host(ids, 40, host)
+    assert dec.status() == 0
+    dec.close()
+    assert regular.shape == (3, shape.vocab)
+    assert float((static - regular).abs().max()) <= 1e-3 and float((host - regular).abs().max()) <= 1e-3
+    assert float(regular.abs().max()) > 0.05
