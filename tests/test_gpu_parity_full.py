@@ -27,7 +27,9 @@ def weights_for(shape):
     return _weights[shape.name]
 
 
-@pytest.mark.parametrize("name", ["c3", "c4", "c5"])
+# the last case is one of Table 2's presets: warm-up layer 1, budget 8 -> 5, and a sequence that ends at the
+# model's last learned position (1024 + 1024 = 2048)
+@pytest.mark.parametrize("name", ["c3", "c4", "c5", "t2-6.7b-5x-cnndm"])
 def test_full_size_sampled_rows(name):
     wl = synth.CONFIGS[name]
     w = weights_for(wl.shape)
@@ -47,7 +49,11 @@ def test_full_size_sampled_rows(name):
     dec.close()
     del dec
     torch.cuda.empty_cache()
-    assert steps == wl.gen_len and layer_steps == wl.gen_len * (wl.max_layers + wl.min_layers) // 2
+    from oracle import skipdecode_oracle as O
+    n_active, _ = O.schedule(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len, wl.shape.n_layers)
+    assert steps == wl.gen_len and layer_steps == sum(n_active)
+    if wl.warmup == 0:
+        assert layer_steps == wl.gen_len * (wl.max_layers + wl.min_layers) // 2
     ref = harness.oracle_run_forced(wl, w, prompts, forced, rows=rows, dtype=torch.float32)
     tol = harness.TOL["bf16"]
     err, strict, near = harness.compare(gpu, ref, tol)
