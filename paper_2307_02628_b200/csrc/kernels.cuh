@@ -156,6 +156,19 @@ layernorm_kernel(const float* __restrict__ x, const T* __restrict__ gamma, const
       v[i] = k < nvec ? reinterpret_cast<const float4*>(xr)[k] : make_float4(0.f, 0.f, 0.f, 0.f);
       s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
     }
+    // bf16 storage: gain and offset as 8-byte vectors, fetched before the reductions so that their latency
+    // hides behind them, and the operand row written as 8-byte vectors (4 hi, 4 lo)
+    constexpr bool kVec = sizeof(T) == 2;
+    const bool vec = kVec && ((reinterpret_cast<uintptr_t>(gamma) | reinterpret_cast<uintptr_t>(beta)) & 7) == 0;
+    uint2 gv[MAXV], bv[MAXV];
+    if (vec) {
+#pragma unroll
+      for (int i = 0; i < MAXV; ++i) {
+        const int k = i * blockDim.x + threadIdx.x;
+        gv[i] = k < nvec ? reinterpret_cast<const uint2*>(gamma)[k] : make_uint2(0u, 0u);
+        bv[i] = k < nvec ? reinterpret_cast<const uint2*>(beta)[k] : make_uint2(0u, 0u);
+      }
+    }
     const float mean = block_sum(s, red) / d;
     float q = 0.f;
 #pragma unroll
@@ -172,10 +185,29 @@ layernorm_kernel(const float* __restrict__ x, const T* __restrict__ gamma, const
       const int k = i * blockDim.x + threadIdx.x;
       if (k < nvec) {
         const float vals[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+        if (vec) {
+          // a bf16 is the upper half of the float with the same value
+          const float g[4] = {__uint_as_float(gv[i].x << 16), __uint_as_float(gv[i].x & 0xffff0000u),
+                              __uint_as_float(gv[i].y << 16), __uint_as_float(gv[i].y & 0xffff0000u)};
+          const float o[4] = {__uint_as_float(bv[i].x << 16), __uint_as_float(bv[i].x & 0xffff0000u),
+                              __uint_as_float(bv[i].y << 16), __uint_as_float(bv[i].y & 0xffff0000u)};
+          uint32_t hi[4], lo[4];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const int c = 4 * k + t;
-          Operand<T>::store(ur, d, c, (vals[t] - mean) * rstd * to_f32(gamma[c]) + to_f32(beta[c]));
+          for (int t = 0; t < 4; ++t) {
+            const float y = (vals[t] - mean) * rstd * g[t] + o[t];
+            const __nv_bfloat16 h = __float2bfloat16_rn(y);
+            hi[t] = __bfloat16_as_ushort(h);
+            lo[t] = __bfloat16_as_ushort(__float2bfloat16_rn(y - __bfloat162float(h)));
+          }
+          uint2* dst = reinterpret_cast<uint2*>(ur);          // row of 2 d bf16: hi | lo
+          dst[k] = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+          dst[(d >> 2) + k] = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+        } else {
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const int c = 4 * k + t;
+            Operand<T>::store(ur, d, c, (vals[t] - mean) * rstd * to_f32(gamma[c]) + to_f32(beta[c]));
+          }
         }
       }
     }
@@ -406,9 +438,24 @@ __global__ void greedy_kernel(const float* __restrict__ logits, int vocab, int32
   const float* row = logits + (size_t)blockIdx.x * vocab;
   float best = -INFINITY;
   int bi = 0x7fffffff;
-  for (int c = threadIdx.x; c < vocab; c += blockDim.x) {
-    const float v = row[c];
-    if (v > best || (v == best && c < bi)) { best = v; bi = c; }
+  if ((vocab & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0) {
+    // 16-byte loads, four in flight per thread: the row is read once and the kernel is latency-bound
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    const int n4 = vocab >> 2;
+#pragma unroll 4
+    for (int c4 = threadIdx.x; c4 < n4; c4 += blockDim.x) {
+      const float4 v = row4[c4];
+      const int c = c4 << 2;                    // a thread's columns increase, so ">" keeps the lowest index of a tie
+      if (v.x > best) { best = v.x; bi = c; }
+      if (v.y > best) { best = v.y; bi = c + 1; }
+      if (v.z > best) { best = v.z; bi = c + 2; }
+      if (v.w > best) { best = v.w; bi = c + 3; }
+    }
+  } else {
+    for (int c = threadIdx.x; c < vocab; c += blockDim.x) {
+      const float v = row[c];
+      if (v > best || (v == best && c < bi)) { best = v; bi = c; }
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
