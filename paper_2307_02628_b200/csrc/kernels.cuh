@@ -130,6 +130,20 @@ __global__ void embed_pos_kernel(const int32_t* __restrict__ ids, const T* __res
   const T* te = tok_emb + (size_t)id * d;
   const T* pe = pos_emb + (size_t)pos * d;
   float* xr = x + (size_t)r * d;
+  if (sizeof(T) == 2 && (d & 3) == 0 && ((reinterpret_cast<uintptr_t>(tok_emb) | reinterpret_cast<uintptr_t>(pos_emb)) & 7) == 0) {
+    // bf16 tables: four elements per 8-byte load (a bf16 is the upper half of the float with the same value)
+    const uint2* te2 = reinterpret_cast<const uint2*>(te);
+    const uint2* pe2 = reinterpret_cast<const uint2*>(pe);
+    for (int k = threadIdx.x; k < (d >> 2); k += blockDim.x) {
+      const uint2 a = te2[k], p = pe2[k];
+      reinterpret_cast<float4*>(xr)[k] =
+          make_float4(__uint_as_float(a.x << 16) + __uint_as_float(p.x << 16),
+                      __uint_as_float(a.x & 0xffff0000u) + __uint_as_float(p.x & 0xffff0000u),
+                      __uint_as_float(a.y << 16) + __uint_as_float(p.y << 16),
+                      __uint_as_float(a.y & 0xffff0000u) + __uint_as_float(p.y & 0xffff0000u));
+    }
+    return;
+  }
   for (int c = threadIdx.x; c < d; c += blockDim.x) xr[c] = to_f32(te[c]) + to_f32(pe[c]);
 }
 
