@@ -72,6 +72,8 @@ CONFIGS = {
     # profiler case: config 4's kernels (same d, heads, batch, prompt, hence the same attention and GEMM
     # launches) on a 2-layer model, so that a counter capture holds a few GB instead of 60
     "c4-2layer": Workload(ModelShape("opt-6.7b-2layer", 2, 4096, 32, 16384, 50272, 2048, "bf16"), 64, 1024, 16, 2, 2),
+    # the same for config 5's launches (batch 256: the tensor-bound GEMM regime)
+    "c5-2layer": Workload(ModelShape("opt-6.7b-2layer", 2, 4096, 32, 16384, 50272, 2048, "bf16"), 256, 256, 16, 2, 2),
 }
 
 

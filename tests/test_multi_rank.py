@@ -30,7 +30,7 @@ def test_two_ranks_report_the_slowest_time_and_the_whole_job_rate():
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0))
         port = s.getsockname()[1]
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:      # never fork a process that already has threads
         out = mgr.dict()
         mp.spawn(_rank, args=(2, port, out), nprocs=2, join=True)
         res = dict(out)
