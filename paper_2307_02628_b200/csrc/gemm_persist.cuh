@@ -23,6 +23,21 @@ constexpr int ACC_COLS = 2 * NB;                 // one accumulator: W.hi in [0,
 constexpr int TMEM_COLS = 2 * ACC_COLS;          // two accumulators = all 512 columns
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/;
 
+// Order in which the CTAs walk over the output tiles.  The CTAs that run at the same time hold
+// consecutive tile numbers, and what they read at the same time they fetch from DRAM once (the rest are
+// L2 hits).  Tiles are therefore numbered in bands of BAND weight tiles, weight tile fastest inside a
+// band: one wave of CTAs then covers about BAND weight tiles x (SMs / BAND) token tiles instead of every
+// weight tile for a single token tile.  A token tile (hi + lo) is twice a weight tile in bytes, so a wave
+// of S CTAs fetches BAND + 2 S / BAND tile units, least near BAND = sqrt(2 S): 16 for 148 SMs.
+constexpr int BAND = 16;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_n, int tiles_m, int& tn, int& tm) {
+  const int band_tiles = BAND * tiles_m;
+  const int band = tile / band_tiles, r = tile - band * band_tiles;
+  const int width = min(BAND, tiles_n - band * BAND);        // the last band may be narrower
+  tm = r / width;
+  tn = band * BAND + (r - tm * width);
+}
+
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -44,6 +59,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb = K / BK;
+  const int tiles_m = tiles_total / tiles_n;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -68,7 +84,9 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
       const int first_tile = blockIdx.x;
       const int early = nkb < STAGES ? nkb : STAGES;
       {
-        const int n0 = (first_tile % tiles_n) * BM;
+        int tn, tm;
+        tile_coords(first_tile, tiles_n, tiles_m, tn, tm);
+        const int n0 = tn * BM;
         for (int i = 0; i < early; ++i) {
           const uint32_t fb = full0 + 8 * i;
           mbar_expect_tx(fb, STAGE_BYTES);
@@ -79,7 +97,9 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
       int it = 0;
       bool ok = true;
       for (int tile = first_tile; tile < tiles_total && ok; tile += gridDim.x) {
-        const int n0 = (tile % tiles_n) * BM, m0 = (tile / tiles_n) * NB;
+        int tn, tm;
+        tile_coords(tile, tiles_n, tiles_m, tn, tm);
+        const int n0 = tn * BM, m0 = tm * NB;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGES, round = it / STAGES;
           const uint32_t fb = full0 + 8 * s;
@@ -137,7 +157,9 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles_total && ok; tile += gridDim.x, ++i) {
       const int buf = i & 1, use = i >> 1;
-      const int n0 = (tile % tiles_n) * BM, m0 = (tile / tiles_n) * NB;
+      int tn, tm;
+      tile_coords(tile, tiles_n, tiles_m, tn, tm);
+      const int n0 = tn * BM, m0 = tm * NB;
       const int n = n0 + quarter * 32 + lane;
       int kv_head = 0, kv_elem = 0;
       __nv_bfloat16* kv_base = nullptr;
