@@ -242,6 +242,8 @@ def gpu_arm(args, wl, rank, world):
         dec.set_option(binding.SD_OPT_GEMM_ISSUERS, args.issuers)
     if args.no_persistent:
         dec.set_option(binding.SD_OPT_GEMM_PERSISTENT, 0)
+    if args.splitk is not None:
+        dec.set_option(binding.SD_OPT_GEMM_SPLITK, args.splitk)
     if args.pdl is not None:
         dec.set_option(binding.SD_OPT_PDL, args.pdl)
     if args.attn_chunk:
@@ -437,6 +439,7 @@ def main():
     ap.add_argument("--select", default="greedy", choices=["greedy", "top-p"],
                     help="token selection in the timed generation loop (the five configurations are greedy)")
     ap.add_argument("--no-persistent", action="store_true", help="SD_OPT_GEMM_PERSISTENT = 0")
+    ap.add_argument("--splitk", type=int, default=None, help="SD_OPT_GEMM_SPLITK (most splits of K under a non-linear epilogue; 0 = off)")
     ap.add_argument("--issuers", type=int, default=0, help="SD_OPT_GEMM_ISSUERS (1 or 2; 0 = library default)")
     ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")

@@ -266,9 +266,14 @@ enum {
                               (bf16 storage, head size 64 or 128); 0: one decode-style block per query row */
   SD_OPT_GEMM_ISSUERS = 9, /* MMA-issuing warps per block of the 128-row GEMM at up to 64 tokens: 1 or 2
                               (2: alternate k-blocks go to two accumulators that the epilogue adds)       */
-  SD_OPT_GEMM_PERSISTENT = 10 /* 1 (default): products with more than 64 tokens and more output tiles than SMs
+  SD_OPT_GEMM_PERSISTENT = 10, /* 1 (default): products with more than 64 tokens and more output tiles than SMs
                               run on the persistent kernel (one block per SM, double-buffered accumulator,
                               epilogue overlapped with the next tile's main loop); 0: one block per tile */
+  SD_OPT_GEMM_SPLITK = 11  /* 0..8, default 8 = the most splits of K for a QKV, fc1 or LM-head product whose output
+                              tiles cover fewer than half of the SMs (every split keeps at least 8 k-blocks of 64);
+                              the partial tiles are parked in the arena and the block that arrives last adds them in
+                              split order and runs the epilogue (results do not depend on arrival order);
+                              0: K is split for the two residual products only */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff

@@ -119,6 +119,11 @@ struct QkvOut {
   RowMap map;
   int packed_kb;     // every epilogue: 0 = W is row-major [N, K]; else W is tile-packed with K/64 tiles per row tile
   const __nv_bfloat16* w_packed;
+  // K split under an epilogue that is not linear (ReLU, rounding into the cache, plain store): every
+  // split parks its partial tile in ws[(tile * splits + split)][token column][weight row] and bumps
+  // ws_count[tile]; the block that arrives last adds the partials in split order and runs the epilogue.
+  float* ws;
+  int* ws_count;     // zero between launches (the last block puts it back)
 };
 
 // Tile-packed weights: [ceil(N/128)][K/64] tiles of 128 rows x 64 columns, each tile stored as
@@ -172,6 +177,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * STAGES, accum_bar = full0 + 16 * STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);   // split K with fix-up: this block arrived last
   long long* col_row = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [NB], QKV epilogue only
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -282,16 +288,71 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     // launch and set-up overlap this kernel's epilogue (earlier would only park its blocks on the
     // SMs for the whole main loop).
     pdl_launch_dependents();
-    if (accum_ok) {
+    // K split under a non-linear epilogue (ISS = 1 only): park the partial tile, count arrivals, and let
+    // the block that arrives last finish the tile from the parked partials
+    const bool fix = ISS == 1 && EPI != EPI_RESIDUAL_F32 && gridDim.z > 1;
+    bool go = accum_ok;
+    if (fix) {
+      // the fix-up meets at a named barrier: all epilogue threads take it or none (a bounded wait may
+      // have expired for some of them only)
+      int all;
+      asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.and.pred p, 1, %2, q;\n selp.b32 %0, 1, 0, p;\n}\n"
+                   : "=r"(all) : "r"((int)accum_ok), "n"(32 * EW) : "memory");
+      go = all != 0;
+    }
+    if (go) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const float b = (bias != nullptr && n < N && (EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
-#pragma unroll 1
       const int c_begin = ((warp - 2) >> 2) * GROUP_COLS;
-      for (int c = c_begin; c < c_begin + GROUP_COLS; c += CW) {
+      const int splits = (int)gridDim.z, tile_id = (int)(blockIdx.y * gridDim.x + blockIdx.x);
+      float* ws_tile = fix ? qo.ws + (size_t)tile_id * splits * (NB * BM) + quarter * 32 + lane : nullptr;
+      bool emit = true;
+      if (fix) {
+        float* mine = ws_tile + (size_t)blockIdx.z * (NB * BM);
+#pragma unroll 1
+        for (int c = c_begin; c < c_begin + GROUP_COLS; c += CW) {
+          uint32_t r[32], rl[32];
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
+          if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < CW; ++j)             // 32 lanes = 32 consecutive weight rows: one 128-byte store per column
+            __stcg(mine + (size_t)(c + j) * BM, __uint_as_float(r[j]) + __uint_as_float(rl[j]));
+        }
+        __threadfence();
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * EW) : "memory");
+        if (threadIdx.x == 64) {
+          const int arrived = atomicAdd(qo.ws_count + tile_id, 1);
+          const int last = arrived == splits - 1;
+          if (last) qo.ws_count[tile_id] = 0;     // every split has arrived: ready for the next launch
+          *last_flag = last;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * EW) : "memory");
+        emit = *last_flag != 0;
+        if (emit) __threadfence();
+      }
+#pragma unroll 1
+      for (int c = c_begin; emit && c < c_begin + GROUP_COLS; c += CW) {
         uint32_t r[32], rl[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
-        if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (fix) {
+          // partials added in split order, so the result does not depend on which block came last; all
+          // loads of one split are in flight together
+#pragma unroll
+          for (int j = 0; j < CW; ++j) { r[j] = 0u; rl[j] = 0u; }
+#pragma unroll 1
+          for (int z = 0; z < splits; ++z) {
+            const float* src = ws_tile + (size_t)z * (NB * BM) + (size_t)c * BM;
+            float t[CW];
+#pragma unroll
+            for (int j = 0; j < CW; ++j) t[j] = __ldcg(src + (size_t)j * BM);
+#pragma unroll
+            for (int j = 0; j < CW; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + t[j]);
+          }
+        } else {
+          if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        }
         if (ISS == 2 && nkb > 1) {                // the second issuer's partial sums
           uint32_t r2[32], rl2[32];
           if (CW == 32) { tmem_ld32(taddr + 2 * NB, r2); tmem_ld32(taddr + 3 * NB, rl2); } else { tmem_ld16(taddr + 2 * NB, r2); tmem_ld16(taddr + 3 * NB, rl2); }
@@ -356,12 +417,18 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+constexpr int kSplitSlots = 160;   // parked partial tiles: tiles x splits of one launch never exceed this
+
 struct TcContext {
   EncodeTiledFn encode = nullptr;
   int ready = 0;
   int sm_count = 148;
   bool pdl = false;      // launch with the programmatic-dependent-launch attribute
   int issuers = 1;       // MMA-issuing warps per block (2 only for token tiles of at most 64)
+  // split K under a non-linear epilogue: parked partial tiles (kSplitSlots of 128 x 128 floats) and arrival counters
+  float* splitk_ws = nullptr;
+  int* splitk_count = nullptr;
+  int splitk = 8;        // most splits of K under a non-linear epilogue; 0: K is split for the residual products only
   // (pointer, rows, cols, box rows) -> tensor map of a row-major bf16 matrix, 64-column boxes, 128-byte swizzle
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
 };
@@ -455,6 +522,16 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   if (epi == EPI_RESIDUAL_F32) {                 // partial sums may be added in any order
     const int tiles = ((N + tc::BM - 1) / tc::BM) * ((M + nb - 1) / nb);
     splits = std::max(1, std::min(kb_total / 4, c.sm_count / tiles));     // one wave: never more blocks than SMs
+  } else if (c.splitk && c.splitk_ws && c.issuers == 1) {
+    // The other epilogues are not linear, so the block that arrives last finishes the tile from parked
+    // partials.  That costs a second pass over the tile: only where fewer than half of the SMs would hold
+    // a block and every split keeps at least 8 k-blocks (the main loop is paced per MMA instruction, so
+    // the time saved is the k-blocks a block no longer issues).
+    const int tiles = ((N + tc::BM - 1) / tc::BM) * ((M + nb - 1) / nb);
+    if (2 * tiles <= c.sm_count)
+      splits = std::max(1, std::min(std::min(std::min(kb_total / 8, c.sm_count / tiles), kSplitSlots / tiles), c.splitk));
+    qo.ws = c.splitk_ws;
+    qo.ws_count = c.splitk_count;
   }
   int kb_per_split = (kb_total + splits - 1) / splits;
   splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split

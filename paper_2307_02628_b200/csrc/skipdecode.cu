@@ -37,7 +37,7 @@ struct Arena {            // byte offsets into the caller's arena
   size_t wp_head;
   bool packable;
   std::vector<int> cap;
-  size_t x, u, qkv, o, y, part_acc, part_ml, counters, row_index, ids, logits, scalars, pad, rows, total;
+  size_t x, u, qkv, o, y, part_acc, part_ml, counters, row_index, ids, logits, scalars, pad, rows, splitk_ws, splitk_count, total;
   int rows_max;
   size_t part_slots;
 };
@@ -191,6 +191,12 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   // batch rows still generating; a GEMM epilogue looks up whole token tiles (up to 127 entries past the
   // row count, results unused), so the array is that much longer than the batch
   A.rows = take(((size_t)c.max_batch + 128) * 4);
+  // bf16 storage: parked partial tiles and arrival counters of the GEMMs that split K under a non-linear epilogue
+  A.splitk_ws = A.splitk_count = 0;
+  if (c.dtype == SD_DTYPE_BF16) {
+    A.splitk_ws = take((size_t)sd::kSplitSlots * 128 * 128 * 4);
+    A.splitk_count = take((size_t)sd::kSplitSlots * 4);
+  }
   A.total = off;
 }
 
@@ -575,6 +581,13 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
       cudaMemsetAsync(h->arena + h->A.counters, 0, (size_t)h->A.rows_max * cfg->n_heads * 4, h->stream) != cudaSuccess) {
     cudaGetLastError(); delete h; return SD_ERR_CUDA;
   }
+  if (cfg->dtype == SD_DTYPE_BF16) {
+    if (cudaMemsetAsync(h->arena + h->A.splitk_count, 0, (size_t)sd::kSplitSlots * 4, h->stream) != cudaSuccess) {
+      cudaGetLastError(); delete h; return SD_ERR_CUDA;
+    }
+    h->tc.splitk_ws = h->at<float>(h->A.splitk_ws);
+    h->tc.splitk_count = h->at<int>(h->A.splitk_count);
+  }
   sd::tc_init(h->tc);
   sd::wide_init(h->wide, h->tc);
   sd::xs_init(h->xs, h->tc);
@@ -861,6 +874,10 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != 1 && value != 2) return SD_ERR_ARG;
       if (value != h->tc.issuers) drop_graphs(h);
       h->tc.issuers = value; return SD_OK;
+    case SD_OPT_GEMM_SPLITK:
+      if (value < 0 || value > 8) return SD_ERR_ARG;
+      if (value != h->tc.splitk) drop_graphs(h);
+      h->tc.splitk = value; return SD_OK;
     case SD_OPT_GEMM_PERSISTENT:
       if ((value != 0) != (h->persist.enabled != 0)) drop_graphs(h);
       h->persist.enabled = value ? 1 : 0; return SD_OK;

@@ -331,6 +331,33 @@ def test_persistent_gemm_in_the_prompt_pass(B, P):
     assert float((runs[1] - runs[0]).abs().max()) <= 2e-3     # same products; the residual adds arrive in another order
 
 
+@pytest.mark.parametrize("d,heads,B", [(1024, 8, 20), (1024, 8, 64), (1536, 12, 33), (1536, 12, 100)])
+def test_split_k_under_nonlinear_epilogues(d, heads, B):
+    # few output tiles and 16 or 24 k-blocks: the QKV (cache-writing), fc1 (ReLU) and LM-head (store) products of
+    # a decode step split K in two or three, park their partial tiles and let the last block finish the tile;
+    # token tiles of 32, 64 and 128
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("splitk-bf16", 2, d, heads, 2048, 640, 64, "bf16")
+    wl = synth.Workload(shape, B, 9, 5, 2, 1, 0)
+    w = synth.make_weights(shape, seed=15, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    rows = synth.sample_rows(B, 6)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced, rows=rows)
+    runs = {}
+    for splitk in (8, 0):
+        for graphs in (1, 0):
+            dec = harness.make_decoder(wl, w)
+            dec.set_option(binding.SD_OPT_GEMM_SPLITK, splitk)
+            dec.set_option(binding.SD_OPT_GRAPHS, graphs)
+            runs[splitk, graphs] = harness.gpu_run_forced(dec, wl, prompts, forced, rows=rows)
+            dec.close()
+            err, strict, near = harness.compare(runs[splitk, graphs], ref, harness.TOL["bf16"])
+            print(f"splitk={splitk} graphs={graphs} d={d} B={B}: max|err|={err:.3e} argmax strict={strict:.4f} near={near:.4f}")
+            assert err <= harness.TOL["bf16"] and near >= 0.99
+    assert float((runs[8, 1] - runs[0, 1]).abs().max()) <= 2e-3     # same products, partial sums added in another order
+    assert float((runs[8, 1] - runs[8, 0]).abs().max()) <= 2e-3
+
+
 @pytest.mark.parametrize("alpha", [2, 3])
 def test_power_law_budget_table(alpha):
     """A caller-supplied budget table (power-law decay with warm-up 1) through sd_schedule_custom."""
