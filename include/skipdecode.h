@@ -268,7 +268,9 @@ enum {
                               (2: alternate k-blocks go to two accumulators that the epilogue adds)       */
   SD_OPT_GEMM_PERSISTENT = 10, /* 1 (default): products with more than 64 tokens and more output tiles than SMs
                               run on the persistent kernel (one block per SM, double-buffered accumulator,
-                              epilogue overlapped with the next tile's main loop); 0: one block per tile */
+                              epilogue overlapped with the next tile's main loop; token tiles of 128, or of 96
+                              where that takes fewer rounds of tiles per block); 2: the same with 128-token
+                              tiles only; 0: one block per tile */
   SD_OPT_GEMM_SPLITK = 11  /* 0..8, default 8 = the most splits of K for a QKV, fc1 or LM-head product whose output
                               tiles cover fewer than half of the SMs (every split keeps at least 8 k-blocks of 64);
                               the partial tiles are parked in the arena and the block that arrives last adds them in

@@ -16,12 +16,13 @@ namespace sd {
 namespace tcp {
 using namespace tc;
 
-constexpr int NB = 128;
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
-constexpr int ACC_COLS = 2 * NB;                 // one accumulator: W.hi in [0, NB), W.lo in [NB, 2 NB)
-constexpr int TMEM_COLS = 2 * ACC_COLS;          // two accumulators = all 512 columns
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/;
+// Token tile NB = 128, or 96 where that needs fewer rounds of tiles per block (config 5's QKV: 96 x 2 = 192
+// tiles of 128 tokens are two rounds for 148 blocks, 96 x 3 = 288 tiles of 96 tokens two rounds of 3/4 the work).
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int TMEM_COLS = 512;                   // two accumulators of 2 NB columns each (all 512 columns at NB = 128)
+__host__ __device__ constexpr int stages(int nb) { return nb >= 128 ? 4 : 5; }
+__host__ __device__ constexpr int stage_bytes(int nb) { return A_BYTES + 2 * nb * BK * 2; }
+__host__ __device__ constexpr int smem_bytes(int nb) { return stages(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
 
 // Order in which the CTAs walk over the output tiles.  The CTAs that run at the same time hold
 // consecutive tile numbers, and what they read at the same time they fetch from DRAM once (the rest are
@@ -42,11 +43,13 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-template <int EPI>
+template <int NB, int EPI>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                        const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                        int tiles_n, int tiles_total, int* __restrict__ status, const QkvOut qo) {
+  constexpr int STAGES = stages(NB), B_BYTES = NB * BK * 2, STAGE_BYTES = stage_bytes(NB);
+  constexpr int ACC_COLS = 2 * NB;               // one accumulator: W.hi in [0, NB), W.lo in [NB, 2 NB)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -164,9 +167,11 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
       int kv_head = 0, kv_elem = 0;
       __nv_bfloat16* kv_base = nullptr;
       if (EPI == EPI_QKV_CACHE) {
-        int b, pos;
-        qo.map.get(m0 + t_epi, b, pos);
-        col_row[t_epi] = (m0 + t_epi < M && pos < qo.cap) ? (long long)b * qo.H * qo.cap + pos : -1;
+        if (t_epi < NB) {
+          int b, pos;
+          qo.map.get(m0 + t_epi, b, pos);
+          col_row[t_epi] = (m0 + t_epi < M && pos < qo.cap) ? (long long)b * qo.H * qo.cap + pos : -1;
+        }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (n >= qo.d && n < N) {
           const int cc = n < 2 * qo.d ? n - qo.d : n - 2 * qo.d;
@@ -226,11 +231,26 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
 
 }  // namespace tcp
 
-struct PersistContext { int ready = 0; int enabled = 1; };
+struct PersistContext { int ready = 0; int enabled = 1; int allow_96 = 1; };
 
 template <int EPI>
 inline bool persist_prepare() {
-  return cudaFuncSetAttribute(tcp::gemm_tc_persist_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tcp::SMEM_BYTES) == cudaSuccess;
+  return cudaFuncSetAttribute(tcp::gemm_tc_persist_kernel<128, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tcp::smem_bytes(128)) == cudaSuccess &&
+         cudaFuncSetAttribute(tcp::gemm_tc_persist_kernel<96, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tcp::smem_bytes(96)) == cudaSuccess;
+}
+template <int NB>
+inline void persist_launch(bool pdl, cudaStream_t st, int sms, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias,
+                           void* out, int ldo, int M, int N, int K, int tiles_n, int total, int epi, int* status, const tc::QkvOut& qo) {
+  const dim3 grid(sms), block(192);
+  constexpr int smem = tcp::smem_bytes(NB);
+  if (epi == EPI_STORE_F32)
+    launch_kernel(pdl, st, tcp::gemm_tc_persist_kernel<NB, EPI_STORE_F32>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  else if (epi == EPI_RELU_T)
+    launch_kernel(pdl, st, tcp::gemm_tc_persist_kernel<NB, EPI_RELU_T>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  else if (epi == EPI_QKV_CACHE)
+    launch_kernel(pdl, st, tcp::gemm_tc_persist_kernel<NB, EPI_QKV_CACHE>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  else
+    launch_kernel(pdl, st, tcp::gemm_tc_persist_kernel<NB, EPI_RESIDUAL_F32>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
 }
 inline void persist_init(PersistContext& p, const TcContext& c) {
   if (!c.ready) return;
@@ -250,25 +270,21 @@ inline bool persist_gemm(PersistContext& p, TcContext& c, cudaStream_t st, const
   if (!p.ready || !p.enabled || !c.ready || K % tc::BK || M <= 64 || N < 1) return false;
   if (epi == EPI_QKV_CACHE && (!qkv_out || qkv_out->d % tc::BM || N != 3 * qkv_out->d)) return false;
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
-  const int tiles_n = (N + tc::BM - 1) / tc::BM, tiles_m = (M + tcp::NB - 1) / tcp::NB;
-  const int total = tiles_n * tiles_m;
-  if (total <= c.sm_count) return false;
+  const int tiles_n = (N + tc::BM - 1) / tc::BM;
+  if (tiles_n * ((M + 127) / 128) <= c.sm_count) return false;
   if (K / tc::BK > 128) return false;       // long main loops hide little behind them (measured: fc2 3 % slower here)
+  // token tile: the one whose tiles take less time per block, counted as rounds of tiles x tokens per tile
+  auto cost = [&](int nb) { return (tiles_n * ((M + nb - 1) / nb) + c.sm_count - 1) / c.sm_count * nb; };
+  const int nb = (p.allow_96 && cost(96) < cost(128)) ? 96 : 128;
+  const int total = tiles_n * ((M + nb - 1) / nb);
   tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
   qo.packed_kb = Wp ? K / tc::BK : 0;
   qo.w_packed = Wp;
   const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
-  const CUtensorMap* mx = tc_map(c, X, M, 2 * K, tcp::NB);
+  const CUtensorMap* mx = tc_map(c, X, M, 2 * K, nb);
   if (!mw || !mx) return false;
-  const dim3 grid(c.sm_count), block(192);
-  if (epi == EPI_STORE_F32)
-    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_STORE_F32>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
-  else if (epi == EPI_RELU_T)
-    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_RELU_T>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
-  else if (epi == EPI_QKV_CACHE)
-    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_QKV_CACHE>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
-  else
-    launch_kernel(c.pdl, st, tcp::gemm_tc_persist_kernel<EPI_RESIDUAL_F32>, grid, block, tcp::SMEM_BYTES, *mw, *mx, bias, out, ldo, M, N, K, tiles_n, total, status, qo);
+  if (nb == 96) persist_launch<96>(c.pdl, st, c.sm_count, mw, mx, bias, out, ldo, M, N, K, tiles_n, total, epi, status, qo);
+  else persist_launch<128>(c.pdl, st, c.sm_count, mw, mx, bias, out, ldo, M, N, K, tiles_n, total, epi, status, qo);
   return true;
 }
 template <typename T>

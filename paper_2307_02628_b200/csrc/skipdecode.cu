@@ -879,8 +879,10 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != h->tc.splitk) drop_graphs(h);
       h->tc.splitk = value; return SD_OK;
     case SD_OPT_GEMM_PERSISTENT:
-      if ((value != 0) != (h->persist.enabled != 0)) drop_graphs(h);
-      h->persist.enabled = value ? 1 : 0; return SD_OK;
+      if (value < 0 || value > 2) return SD_ERR_ARG;
+      drop_graphs(h);
+      h->persist.enabled = value ? 1 : 0;
+      h->persist.allow_96 = value == 1 ? 1 : 0; return SD_OK;
     case SD_OPT_PREFILL_ATTN:
       h->opt_prefill = value ? 1 : 0; return SD_OK;
     case SD_OPT_WEIGHT_TILES:

@@ -331,6 +331,30 @@ def test_persistent_gemm_in_the_prompt_pass(B, P):
     assert float((runs[1] - runs[0]).abs().max()) <= 2e-3     # same products; the residual adds arrive in another order
 
 
+def test_persistent_gemm_with_96_token_tiles():
+    # 2400 prompt tokens and 8 to 24 weight tiles per product: 96-token tiles take fewer rounds per block than
+    # 128-token tiles, so the QKV, out-proj, fc1 and fc2 products of the prompt pass run on them (25 token tiles,
+    # none ragged); at 160 rows per decode step so does the LM head (100 weight tiles, second token tile ragged)
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("persist96-bf16", 2, 1024, 8, 1024, 12800, 32, "bf16")
+    wl = synth.Workload(shape, 160, 15, 3, 2, 1, 0)
+    w = synth.make_weights(shape, seed=16, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    rows = synth.sample_rows(wl.batch, 6)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced, rows=rows)
+    runs = {}
+    for mode in (1, 2, 0):
+        dec = harness.make_decoder(wl, w)
+        dec.set_option(binding.SD_OPT_GEMM_PERSISTENT, mode)
+        runs[mode] = harness.gpu_run_forced(dec, wl, prompts, forced, rows=rows)
+        dec.close()
+        err, strict, near = harness.compare(runs[mode], ref, harness.TOL["bf16"])
+        print(f"persistent={mode}: max|err|={err:.3e} argmax strict={strict:.4f} near={near:.4f}")
+        assert err <= harness.TOL["bf16"] and near >= 0.99
+    assert float((runs[1] - runs[2]).abs().max()) <= 2e-3
+    assert float((runs[1] - runs[0]).abs().max()) <= 2e-3
+
+
 @pytest.mark.parametrize("d,heads,B", [(1024, 8, 20), (1024, 8, 64), (1536, 12, 33), (1536, 12, 100)])
 def test_split_k_under_nonlinear_epilogues(d, heads, B):
     # few output tiles and 16 or 24 k-blocks: the QKV (cache-writing), fc1 (ReLU) and LM-head (store) products of
