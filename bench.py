@@ -236,10 +236,6 @@ def gpu_arm(args, wl, rank, world):
         dec.set_option(binding.SD_OPT_GRAPHS, 0)
     if args.gemm_mode:
         dec.set_option(binding.SD_OPT_GEMM, args.gemm_mode)
-    if args.cluster:
-        dec.set_option(binding.SD_OPT_CLUSTER, args.cluster)
-    if args.issuers:
-        dec.set_option(binding.SD_OPT_GEMM_ISSUERS, args.issuers)
     if args.no_persistent:
         dec.set_option(binding.SD_OPT_GEMM_PERSISTENT, 0)
     if args.splitk is not None:
@@ -434,13 +430,11 @@ def main():
     ap.add_argument("--max-gen-steps", type=int, default=0,
                     help="run only the first N decode steps of each pass (for short profiler captures)")
     ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA graph replay (profiler runs)")
-    ap.add_argument("--gemm-mode", type=int, default=0, help="SD_OPT_GEMM (0 automatic, 1 CUDA cores, 2 128-row kernel)")
-    ap.add_argument("--cluster", type=int, default=0, help="SD_OPT_CLUSTER (0 automatic)")
+    ap.add_argument("--gemm-mode", type=int, default=0, help="SD_OPT_GEMM (0 automatic, 1 CUDA cores)")
     ap.add_argument("--select", default="greedy", choices=["greedy", "top-p"],
                     help="token selection in the timed generation loop (the five configurations are greedy)")
     ap.add_argument("--no-persistent", action="store_true", help="SD_OPT_GEMM_PERSISTENT = 0")
     ap.add_argument("--splitk", type=int, default=None, help="SD_OPT_GEMM_SPLITK (most splits of K under a non-linear epilogue; 0 = off)")
-    ap.add_argument("--issuers", type=int, default=0, help="SD_OPT_GEMM_ISSUERS (1 or 2; 0 = library default)")
     ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")

@@ -130,11 +130,12 @@ int sd_schedule_compute(int n_layers, int max_layers, int min_layers, int warmup
  *     n_active[g] = round_half_up(min_layers + (max_layers - min_layers) * (1 - t)^alpha),  t = g / (gen_len - 1)
  * with an integer exponent 1 <= alpha <= 8, computed in integers; alpha = 1 is the linear schedule and
  * alpha > 1 never exceeds it, so a plan sized for the linear schedule holds every alpha.
- * Errors: SD_ERR_ARG. */
+ * Errors: SD_ERR_ARG, also when (gen_len - 1)^alpha * 2 (max_layers - min_layers) would not fit the
+ * 128-bit integers the rounding is done in (gen_len beyond about 2^14 at alpha = 8). */
 int sd_schedule_power_compute(int n_layers, int max_layers, int min_layers, int warmup, int gen_len, int alpha,
                               int32_t *n_active, int32_t *top_begin);
 
-/* Installs a caller-supplied budget table ("this function can adopt multiple forms", Section 2.3):
+/* Installs a caller-supplied budget table (Section 2.3 allows budget functions other than the linear decay):
  * n_active: host, gen_len int32, non-increasing (Section 2.2), warmup < n_active[g] <= n_layers.
  * The layers that run at g are [0, warmup) and [n_layers - (n_active[g] - warmup), n_layers).
  * top_begin: host, gen_len int32, may be NULL.  Same effects and capacity rule as sd_schedule.
@@ -252,20 +253,14 @@ int sd_launch_count(sd_handle *h, int64_t *launches);
 enum {
   SD_OPT_GRAPHS = 1,       /* 1 (default): replay one CUDA graph per step shape; 0: plain launches */
   SD_OPT_ATTN_CHUNK = 2,   /* keys per split of the decode attention (multiple of 32); 0 = automatic */
-  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (128-row weight-stationary tensor-core kernel, else
-                              CUDA cores); 1 = CUDA cores only; 2 = 128-row kernel; 3 = 256-row cluster
-                              kernel; 4 = token-stationary kernel (up to 64 tokens).  3 and 4 are measured
-                              alternatives that are slower at the shapes tried; they fall back to 2.    */
+  SD_OPT_GEMM = 3,         /* bf16 mode: 0 = automatic (tensor-core kernels, CUDA cores for shapes they do
+                              not take); 1 = CUDA cores only; 2 = same as 0                              */
   SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
   SD_OPT_PDL = 5,          /* programmatic dependent launch: mask of kernel classes (1 << SD_K_*) whose
                               kernels may begin before their predecessor ends; 0 = none             */
-  SD_OPT_CLUSTER = 6,      /* blocks per cluster that split K in the cluster GEMMs: 0 = automatic, 1..4
-                              (the token-stationary kernel uses 1 or 2)                               */
   SD_OPT_WEIGHT_TILES = 7, /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
   SD_OPT_PREFILL_ATTN = 8, /* 1 (default): sd_prefill's causal attention runs as 64x64 tensor-core tiles
                               (bf16 storage, head size 64 or 128); 0: one decode-style block per query row */
-  SD_OPT_GEMM_ISSUERS = 9, /* MMA-issuing warps per block of the 128-row GEMM at up to 64 tokens: 1 or 2
-                              (2: alternate k-blocks go to two accumulators that the epilogue adds)       */
   SD_OPT_GEMM_PERSISTENT = 10, /* 1 (default): products with more than 64 tokens and more output tiles than SMs
                               run on the persistent kernel (one block per SM, double-buffered accumulator,
                               epilogue overlapped with the next tile's main loop; token tiles of 128, or of 96

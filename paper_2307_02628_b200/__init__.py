@@ -3,4 +3,4 @@
 Importing the package loads nothing; `paper_2307_02628_b200.binding` opens the
 shared library on first use and raises if it has not been built.
 """
-__all__ = ["binding", "synth", "build"]
+__all__ = ["binding", "shapes", "synth", "build"]

@@ -11,13 +11,13 @@ import os
 
 import torch
 
-from . import synth
+from .shapes import ModelShape, storage_dtype
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libskipdecode.so")
 _lib = None
 
 SD_OK, SD_ERR_ARG, SD_ERR_STATE, SD_ERR_POSITION, SD_ERR_CAPACITY, SD_ERR_CUDA, SD_ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
-SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING, SD_OPT_PDL, SD_OPT_CLUSTER, SD_OPT_WEIGHT_TILES, SD_OPT_PREFILL_ATTN, SD_OPT_GEMM_ISSUERS, SD_OPT_GEMM_PERSISTENT, SD_OPT_GEMM_SPLITK = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11
+SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING, SD_OPT_PDL, SD_OPT_WEIGHT_TILES, SD_OPT_PREFILL_ATTN, SD_OPT_GEMM_PERSISTENT, SD_OPT_GEMM_SPLITK = 1, 2, 3, 4, 5, 7, 8, 10, 11
 KERNEL_CLASSES = ("embed", "layernorm", "gemm_qkv", "kv_append", "attention", "lm_head", "gemm_out", "gemm_fc1", "gemm_fc2")
 
 EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_schedule_power_compute",
@@ -99,7 +99,7 @@ def _check(code: int, where: str):
         raise SdError(code, where)
 
 
-def make_config(shape: synth.ModelShape, max_batch: int, max_prompt: int, max_gen: int) -> SdConfig:
+def make_config(shape: ModelShape, max_batch: int, max_prompt: int, max_gen: int) -> SdConfig:
     return SdConfig(shape.n_layers, shape.d_model, shape.n_heads, shape.d_ffn, shape.vocab, shape.max_pos,
                     max_batch, max_prompt, max_gen, 0 if shape.dtype == "fp32" else 1, 1e-5)
 
@@ -136,12 +136,12 @@ def arena_bytes(cfg: SdConfig, plan: SdPlan) -> int:
 class Decoder:
     """A handle of the CUDA library plus the device buffers it was given.
 
-    weights: the dict layout of `synth.make_weights` (CPU or CUDA tensors in the
+    weights: a dict {tok_emb, pos_emb, lnf_g, lnf_b, [lm_head], layers: [{ln1_g, ..., b_fc2}]} (CPU or CUDA tensors in the
     configuration's storage type); they are moved to `device` and kept alive here.
     plan: (max_layers, min_layers, warmup, gen_len) the KV caches are sized for.
     """
 
-    def __init__(self, shape: synth.ModelShape, weights: dict, max_batch: int, max_prompt: int, max_gen: int,
+    def __init__(self, shape: ModelShape, weights: dict, max_batch: int, max_prompt: int, max_gen: int,
                  plan=None, full_capacity: bool = False, device: str = "cuda:0", stream=None):
         L = lib()
         if not torch.cuda.is_available():
@@ -153,7 +153,7 @@ class Decoder:
         self.arena_bytes = arena_bytes(self.cfg, self.plan)
         torch.cuda.set_device(self.device)
         self.stream = stream if stream is not None else torch.cuda.Stream(device=self.device)
-        dt = synth.storage_dtype(shape)
+        dt = storage_dtype(shape)
         self._keep = []
 
         def dev(t):

@@ -280,9 +280,9 @@ inline bool persist_gemm(PersistContext& p, TcContext& c, cudaStream_t st, const
   tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
   qo.packed_kb = Wp ? K / tc::BK : 0;
   qo.w_packed = Wp;
-  const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);
-  const CUtensorMap* mx = tc_map(c, X, M, 2 * K, nb);
-  if (!mw || !mx) return false;
+  CUtensorMap mw_v, mx_v;
+  const CUtensorMap *mw = &mw_v, *mx = &mx_v;
+  if (!tc_map(c, W, N, K, tc::BM, &mw_v) || !tc_map(c, X, M, 2 * K, nb, &mx_v)) return false;
   if (nb == 96) persist_launch<96>(c.pdl, st, c.sm_count, mw, mx, bias, out, ldo, M, N, K, tiles_n, total, epi, status, qo);
   else persist_launch<128>(c.pdl, st, c.sm_count, mw, mx, bias, out, ldo, M, N, K, tiles_n, total, epi, status, qo);
   return true;

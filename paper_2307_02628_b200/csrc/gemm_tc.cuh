@@ -4,7 +4,7 @@
 //
 // The weight's output dimension sits on the MMA M axis (D^T = W X^T): a CTA owns 128 rows
 // of W, so tiles are full even when the token count M is 16..256, which becomes the MMA N.
-// Operands reach shared memory by TMA (128-byte swizzle, K-major, no multicast), the
+// Operands reach shared memory by TMA (128-byte swizzle, K-major; every CTA loads its own tiles), the
 // accumulator lives in tensor memory, and one thread issues tcgen05.mma.  Warp roles:
 // warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue (each
 // reads its own quarter of the 128 TMEM lanes).  K can be split over blockIdx.z for the
@@ -146,25 +146,19 @@ __device__ __forceinline__ void load_w_tile(uint32_t dst, const CUtensorMap* map
 // mod 4, so there are four warps per group; with two groups each takes half of the token columns,
 // which halves the serial part of the epilogue (loads from tensor memory, then one store per column).
 __host__ __device__ constexpr int epi_warps(int nb) { return nb >= 32 ? 8 : 4; }
-__host__ __device__ constexpr int block_threads(int nb, int iss) { return 64 + 32 * epi_warps(nb) + 32 * (iss - 1); }
+__host__ __device__ constexpr int block_threads(int nb) { return 64 + 32 * epi_warps(nb); }
 __host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
 __host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
 
-// ISS = 2: a second MMA-issuing warp (warp 6).  The two issuers take alternate k-blocks into
-// accumulators of their own (tensor-memory columns [0, 2 NB) and [2 NB, 4 NB)); the epilogue adds them.
-template <int NB, int EPI, int ISS = 1>
-__global__ void __launch_bounds__(block_threads(NB, ISS), 1)
+template <int NB, int EPI>
+__global__ void __launch_bounds__(block_threads(NB), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                int kb_per_split, int* __restrict__ status, const QkvOut qo) {
-  // With two issuers the stage count is even, so that a stage always belongs to the same issuer (k-block
-  // i, stage i % STAGES and issuer i & 1 then agree in parity).  A phase-parity wait is only safe for a
-  // thread that has itself consumed the stage's previous round: another thread, one round ahead of a
-  // slower consumer, would take the barrier's still-incomplete phase for the one before it.
-  constexpr int STAGES = ISS == 2 ? (stages_for(NB) & ~1) : stages_for(NB);
+  constexpr int STAGES = stages_for(NB);
   constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
-  constexpr int TMEM_COLS = 2 * NB * ISS;        // per issuer: W.hi in columns [0, NB), W.lo in [NB, 2 NB); a power of two >= 32
+  constexpr int TMEM_COLS = 2 * NB;              // W.hi in columns [0, NB), W.lo in [NB, 2 NB); a power of two >= 32
   constexpr int EW = epi_warps(NB);              // epilogue warps: 4, or 8 = two groups that split the columns
   constexpr int GROUP_COLS = NB / (EW / 4);      // token columns per group of four warps
   constexpr int CW = GROUP_COLS < 32 ? 16 : 32;  // accumulator columns read per tcgen05.ld
@@ -188,7 +182,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    mbar_init(accum_bar, (ISS == 2 && nkb > 1) ? 2 : 1);        // one arrival per issuer that has k-blocks
+    mbar_init(accum_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -237,16 +231,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
       }
     }
-  } else if (warp == 1 || (ISS == 2 && warp == 2 + EW)) {
+  } else if (warp == 1) {
     if (lane == 0) {
-      const int w = warp == 1 ? 0 : 1;            // which issuer
       // The hi tile (NB rows) and the lo tile (NB rows) sit back to back in the stage, so they are
       // one K-major operand of 2 NB rows: a single MMA of N = 2 NB per k-step puts W.hi and W.lo
       // side by side in tensor memory (the epilogue adds the halves).  One wide instruction
       // instead of two narrow ones: at these sizes the MMA pipe is paced per instruction.
       constexpr uint32_t idesc = instr_desc(2 * NB);
       bool ok = true;
-      for (int i = w; i < nkb && ok; i += ISS) {
+      for (int i = 0; i < nkb && ok; ++i) {
         const int s = i % STAGES, round = i / STAGES;
         ok = mbar_wait(full0 + 8 * s, round & 1, abort_flag, status);
         if (!ok) break;
@@ -255,10 +248,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const uint64_t a_desc = smem_desc(a_addr), b_desc = smem_desc(a_addr + A_BYTES);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k)     // 32 bytes further along K inside the swizzle row
-          umma(tmem_base + (uint32_t)(w * 2 * NB), a_desc + 2 * k, b_desc + 2 * k, idesc, (i > w || k > 0) ? 1u : 0u);
+          umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
         umma_commit(empty0 + 8 * s);              // the stage is free once these MMAs have read it
       }
-      if (ok && (w == 0 || nkb > 1)) umma_commit(accum_bar);   // this issuer's accumulator is complete
+      if (ok) umma_commit(accum_bar);             // the accumulator is complete
     }
   } else {
     pdl_wait();                                   // bias aside, the epilogue reads and writes buffers earlier kernels own
@@ -288,9 +281,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     // launch and set-up overlap this kernel's epilogue (earlier would only park its blocks on the
     // SMs for the whole main loop).
     pdl_launch_dependents();
-    // K split under a non-linear epilogue (ISS = 1 only): park the partial tile, count arrivals, and let
+    // K split under a non-linear epilogue: park the partial tile, count arrivals, and let
     // the block that arrives last finish the tile from the parked partials
-    const bool fix = ISS == 1 && EPI != EPI_RESIDUAL_F32 && gridDim.z > 1;
+    const bool fix = EPI != EPI_RESIDUAL_F32 && gridDim.z > 1;
     bool go = accum_ok;
     if (fix) {
       // the fix-up meets at a named barrier: all epilogue threads take it or none (a bounded wait may
@@ -353,16 +346,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         }
-        if (ISS == 2 && nkb > 1) {                // the second issuer's partial sums
-          uint32_t r2[32], rl2[32];
-          if (CW == 32) { tmem_ld32(taddr + 2 * NB, r2); tmem_ld32(taddr + 3 * NB, rl2); } else { tmem_ld16(taddr + 2 * NB, r2); tmem_ld16(taddr + 3 * NB, rl2); }
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-          for (int j = 0; j < CW; ++j) {
-            r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
-            rl[j] = __float_as_uint(__uint_as_float(rl[j]) + __uint_as_float(rl2[j]));
-          }
-        }
         if (n < N) {
 #pragma unroll
           for (int j = 0; j < CW; ++j) {
@@ -424,7 +407,6 @@ struct TcContext {
   int ready = 0;
   int sm_count = 148;
   bool pdl = false;      // launch with the programmatic-dependent-launch attribute
-  int issuers = 1;       // MMA-issuing warps per block (2 only for token tiles of at most 64)
   // split K under a non-linear epilogue: parked partial tiles (kSplitSlots of 128 x 128 floats) and arrival counters
   float* splitk_ws = nullptr;
   int* splitk_count = nullptr;
@@ -435,10 +417,7 @@ struct TcContext {
 
 template <int NB, int EPI>
 inline bool tc_prepare() {
-  if (NB <= 64 &&
-      cudaFuncSetAttribute(tc::gemm_tc_kernel<NB, EPI, (NB <= 64 ? 2 : 1)>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(NB)) != cudaSuccess)
-    return false;
-  return cudaFuncSetAttribute(tc::gemm_tc_kernel<NB, EPI, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(NB)) == cudaSuccess;
+  return cudaFuncSetAttribute(tc::gemm_tc_kernel<NB, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(NB)) == cudaSuccess;
 }
 template <int NB>
 inline bool tc_prepare_nb() {
@@ -469,10 +448,12 @@ inline void tc_init(TcContext& c) {
 }
 inline void tc_destroy(TcContext& c) { c.maps.clear(); c.ready = 0; }
 
-inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int cols, int box_rows) {
+// Looks the map up (or encodes it) and copies it into *out: the cache may evict entries on a later call, so
+// callers keep no pointer into it.
+inline bool tc_map(TcContext& c, const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
   auto key = std::make_tuple(ptr, rows, cols, box_rows);
   auto it = c.maps.find(key);
-  if (it != c.maps.end()) return &it->second;
+  if (it != c.maps.end()) { *out = it->second; return true; }
   CUtensorMap m;
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
@@ -481,25 +462,27 @@ inline const CUtensorMap* tc_map(TcContext& c, const void* ptr, int rows, int co
   if (c.encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return nullptr;
+    return false;
   if (c.maps.size() > 4096) c.maps.clear();
-  return &c.maps.emplace(key, m).first->second;
+  c.maps.emplace(key, m);
+  *out = m;
+  return true;
 }
 
-template <int NB, int ISS>
+template <int NB>
 inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CUtensorMap* mx, const __nv_bfloat16* bias, void* out,
                       int ldo, int M, int N, int K, int kb_per_split, int splits, int epi, int* status, const tc::QkvOut& qo) {
   dim3 grid((N + tc::BM - 1) / tc::BM, (M + NB - 1) / NB, splits);
-  const dim3 block(tc::block_threads(NB, ISS));
+  const dim3 block(tc::block_threads(NB));
   const int smem = tc::smem_bytes(NB);
   if (epi == EPI_STORE_F32)
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_STORE_F32, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_STORE_F32>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else if (epi == EPI_RELU_T)
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RELU_T, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RELU_T>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else if (epi == EPI_QKV_CACHE)
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_QKV_CACHE, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_QKV_CACHE>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   else
-    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32, ISS>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
+    launch_kernel(pdl, st, tc::gemm_tc_kernel<NB, EPI_RESIDUAL_F32>, grid, block, smem, *mw, *mx, bias, out, ldo, M, N, K, kb_per_split, status, qo);
   return true;
 }
 
@@ -514,15 +497,15 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   qo.w_packed = Wp;
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
   const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
-  const CUtensorMap* mw = tc_map(c, W, N, K, tc::BM);      // unused by the kernel when the packed copy is read
-  const CUtensorMap* mx = tc_map(c, X, M, 2 * K, nb);
-  if (!mw || !mx) return false;
+  CUtensorMap mw_v, mx_v;
+  const CUtensorMap *mw = &mw_v, *mx = &mx_v;                 // W's map is unused by the kernel when the packed copy is read
+  if (!tc_map(c, W, N, K, tc::BM, &mw_v) || !tc_map(c, X, M, 2 * K, nb, &mx_v)) return false;
   const int kb_total = (K + tc::BK - 1) / tc::BK;
   int splits = 1;
   if (epi == EPI_RESIDUAL_F32) {                 // partial sums may be added in any order
     const int tiles = ((N + tc::BM - 1) / tc::BM) * ((M + nb - 1) / nb);
     splits = std::max(1, std::min(kb_total / 4, c.sm_count / tiles));     // one wave: never more blocks than SMs
-  } else if (c.splitk && c.splitk_ws && c.issuers == 1) {
+  } else if (c.splitk && c.splitk_ws) {
     // The other epilogues are not linear, so the block that arrives last finishes the tile from parked
     // partials.  That costs a second pass over the tile: only where fewer than half of the SMs would hold
     // a block and every split keeps at least 8 k-blocks (the main loop is paced per MMA instruction, so
@@ -535,18 +518,11 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   }
   int kb_per_split = (kb_total + splits - 1) / splits;
   splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split
-  if (c.issuers == 2 && nb <= 64) {
-    switch (nb) {
-      case 16: return tc_launch<16, 2>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-      case 32: return tc_launch<32, 2>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-      default: return tc_launch<64, 2>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    }
-  }
   switch (nb) {
-    case 16: return tc_launch<16, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    case 32: return tc_launch<32, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    case 64: return tc_launch<64, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
-    default: return tc_launch<128, 1>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 16: return tc_launch<16>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 32: return tc_launch<32>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    case 64: return tc_launch<64>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
+    default: return tc_launch<128>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
   }
 }
 template <typename T>

@@ -15,8 +15,6 @@
 
 #include "kernels.cuh"
 #include "gemm_tc.cuh"
-#include "gemm_wide.cuh"
-#include "gemm_xs.cuh"
 #include "gemm_persist.cuh"
 #include "sample.cuh"
 #include "attn_prefill.cuh"
@@ -79,8 +77,6 @@ struct sd_handle {
   double k_ms[SD_K_COUNT] = {};
   int64_t k_launches[SD_K_COUNT] = {};
   sd::TcContext tc;
-  sd::WideContext wide;
-  sd::XsContext xs;
   sd::PersistContext persist;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(arena + off); }
@@ -119,6 +115,18 @@ int budget_at(int mx, int mn, int g, int G) {
 // Power-law variant (Section 2.3 names it as another possible decay): min + (max - min) (1 - t)^alpha
 // with t = g / (G - 1) and an integer exponent, rounded to nearest with halves up, in integers:
 // min + floor((2 D (G-1-g)^alpha + (G-1)^alpha) / (2 (G-1)^alpha)).  alpha = 1 is the linear schedule.
+// True when 2 (max - min) (G-1)^alpha + (G-1)^alpha fits the 128-bit arithmetic below with room to spare.
+bool power_args_fit(int mx, int mn, int G, int alpha) {
+  if (G <= 2) return true;
+  const unsigned __int128 limit = (((unsigned __int128)1) << 124) / (unsigned __int128)(2 * (mx - mn) + 2);
+  unsigned __int128 den = 1;
+  for (int i = 0; i < alpha; ++i) {
+    if (den > limit / (unsigned)(G - 1)) return false;
+    den *= (unsigned)(G - 1);
+  }
+  return true;
+}
+
 int budget_power_at(int mx, int mn, int g, int G, int alpha) {
   if (G == 1) return mx;
   const unsigned __int128 den1 = G - 1, num1 = G - 1 - g;
@@ -247,8 +255,6 @@ void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_of
   Lc.begin(cls);
   bool done = false;
   if (std::is_same<T, bf16>::value && h->opt_gemm != 1) {
-    if (h->opt_gemm == 4) done = sd::xs_gemm(h->xs, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp, h->wide.force_cluster);
-    if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
     if (!done) done = sd::persist_gemm(h->persist, h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
     if (!done) done = sd::tc_gemm(h->tc, h->stream, A, W, bias, M, N, K, out, ldo, epi, h->status(), nullptr, Wp);
   }
@@ -279,8 +285,6 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
   h->tc.pdl = pdl_for(h, SD_K_GEMM_QKV);
   Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
-  if (h->opt_gemm == 4) done = sd::xs_gemm(h->xs, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp, h->wide.force_cluster);
-  if (h->opt_gemm == 3) done = sd::wide_gemm(h->wide, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (!done) done = sd::persist_gemm(h->persist, h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (!done) done = sd::tc_gemm(h->tc, h->stream, u, W, bias, rows, 3 * d, d, qkv, 3 * d, sd::EPI_QKV_CACHE, h->status(), &qo, Wp);
   if (done) Lc.end(); else Lc.cancel();
@@ -440,7 +444,8 @@ template <typename T>
 int run_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_logits) {
   Launcher Lc{h, h->opt_timing != 0, h->at<float>(h->A.part_acc), h->at<float>(h->A.part_ml)};
   const int L = h->cfg.n_layers;
-  const int per = std::max(1, kPrefillTokens / P);
+  // whole batch rows per pass, from the rows the activation buffers were carved for (P <= max_prompt <= rows_max)
+  const int per = std::max(1, h->A.rows_max / P);
   for (int b0 = 0; b0 < B; b0 += per) {
     const int nb = std::min(per, B - b0), rows = nb * P;
     sd::RowMap map{P, b0, 0, nullptr, nullptr, h->d_pad()};
@@ -589,8 +594,6 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
     h->tc.splitk_count = h->at<int>(h->A.splitk_count);
   }
   sd::tc_init(h->tc);
-  sd::wide_init(h->wide, h->tc);
-  sd::xs_init(h->xs, h->tc);
   sd::persist_init(h->persist, h->tc);
   if (h->tc.ready && h->A.packable) {            // tile-packed copies of the matrices, made once
     const int d = cfg->d_model, f = cfg->d_ffn;
@@ -635,7 +638,7 @@ int sd_schedule(sd_handle* h, int mx, int mn, int w, int G, int32_t* n_active, i
 }
 
 int sd_schedule_power_compute(int n_layers, int mx, int mn, int w, int G, int alpha, int32_t* n_active, int32_t* top_begin) {
-  if (!valid_schedule_args(n_layers, mx, mn, w, G) || alpha < 1 || alpha > 8) return SD_ERR_ARG;
+  if (!valid_schedule_args(n_layers, mx, mn, w, G) || alpha < 1 || alpha > 8 || !power_args_fit(mx, mn, G, alpha)) return SD_ERR_ARG;
   for (int g = 0; g < G; ++g) {
     const int n = budget_power_at(mx, mn, g, G, alpha);
     if (n_active) n_active[g] = n;
@@ -863,17 +866,9 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != 0 && (value < kMinChunk || value % kMinChunk)) return SD_ERR_ARG;
       h->opt_chunk = value; return SD_OK;
     case SD_OPT_GEMM:
-      if (value < 0 || value > 4) return SD_ERR_ARG;
+      if (value < 0 || value > 2) return SD_ERR_ARG;
       if (value != h->opt_gemm) drop_graphs(h);
       h->opt_gemm = value; return SD_OK;
-    case SD_OPT_CLUSTER:
-      if (value < 0 || value > sd::tcw::MAX_CLUSTER) return SD_ERR_ARG;
-      if (value != h->wide.force_cluster) drop_graphs(h);
-      h->wide.force_cluster = value; return SD_OK;
-    case SD_OPT_GEMM_ISSUERS:
-      if (value != 1 && value != 2) return SD_ERR_ARG;
-      if (value != h->tc.issuers) drop_graphs(h);
-      h->tc.issuers = value; return SD_OK;
     case SD_OPT_GEMM_SPLITK:
       if (value < 0 || value > 8) return SD_ERR_ARG;
       if (value != h->tc.splitk) drop_graphs(h);

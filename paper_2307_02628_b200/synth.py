@@ -26,21 +26,7 @@ from dataclasses import dataclass, replace
 
 import torch
 
-
-@dataclass(frozen=True)
-class ModelShape:
-    name: str
-    n_layers: int
-    d_model: int
-    n_heads: int
-    d_ffn: int
-    vocab: int
-    max_pos: int
-    dtype: str  # "fp32" | "bf16": storage type of weights, GEMM operands and KV cache
-
-    @property
-    def head_dim(self) -> int:
-        return self.d_model // self.n_heads
+from .shapes import ModelShape, storage_dtype  # noqa: F401  (re-exported)
 
 
 @dataclass(frozen=True)
@@ -100,10 +86,6 @@ def _normal(seed: int, name: str, shape, std: float, dtype: torch.dtype) -> torc
     t = torch.empty(shape, dtype=torch.float32)
     t.normal_(0.0, std, generator=g)
     return t.to(dtype)
-
-
-def storage_dtype(shape: ModelShape) -> torch.dtype:
-    return torch.float32 if shape.dtype == "fp32" else torch.bfloat16
 
 
 def make_weights(shape: ModelShape, seed: int = 0, std: float = 0.02,

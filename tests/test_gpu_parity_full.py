@@ -1,8 +1,8 @@
 """Parity at the full sizes of configurations 3-5, in the launch configuration the benchmark
 times (CUDA graphs on, automatic attention split, tensor-core GEMMs).
 
-The GPU runs the whole batch; the oracle evaluates sampled batch rows (first, last) at the
-full model shape in one layer-major pass of the definition, in fp32 on the same bf16-rounded
+The GPU runs the whole batch; the oracle evaluates sampled batch rows (first, last and one inside
+every 96- and 128-token tile the GEMMs cut the batch into) at the full model shape in one layer-major pass of the definition, in fp32 on the same bf16-rounded
 weights.  Rows are independent, so this checks complete outputs of those rows at every step.
 Both sides consume the same seeded token ids at every step.
 """
@@ -17,6 +17,19 @@ from paper_2307_02628_b200 import binding, synth
 pytestmark = pytest.mark.gpu
 
 _weights = {}
+
+
+def rows_covering_token_tiles(batch: int) -> list:
+    """First and last row plus a seeded row in every interval between consecutive multiples of 96 and 128, so
+    that each token tile of either width has a compared row: 4 rows at batch 256, 2 at batch 64 and below."""
+    import random
+    rng = random.Random(2)
+    cuts = sorted({0, batch} | {c for t in (96, 128) for c in range(t, batch, t)})
+    rows = {0, batch - 1}
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        if not any(lo <= r < hi for r in rows):
+            rows.add(rng.randrange(lo, hi))
+    return sorted(rows)
 
 
 def weights_for(shape):
@@ -41,7 +54,7 @@ def test_full_size_sampled_rows(name):
     free, _ = torch.cuda.mem_get_info()
     if need + wbytes + (3 << 30) > free:
         pytest.skip(f"{name} needs {(need + wbytes) / 2**30:.0f} GiB, {free / 2**30:.0f} GiB free on this GPU")
-    rows = synth.sample_rows(wl.batch, 2)
+    rows = rows_covering_token_tiles(wl.batch)
     prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
     dec = harness.make_decoder(wl, w)
     gpu = harness.gpu_run_forced(dec, wl, prompts, forced, rows=rows)

@@ -101,3 +101,13 @@ def test_config_validation():
                                                  (24, 16, 8, 1, 2047, 4), (12, 12, 4, 0, 1, 2), (12, 12, 4, 0, 2, 8)])
 def test_power_law_schedule_is_bit_exact_with_the_oracle(L, mx, mn, w, G, alpha):
     assert binding.schedule_power_compute(L, mx, mn, w, G, alpha) == tuple(O.schedule_power(mx, mn, w, G, L, alpha))
+
+
+def test_power_law_schedule_rejects_what_its_integers_cannot_hold():
+    # (G-1)^8 * 2 (max - min) passes 2^124 near G = 2^15: refused instead of wrapping around
+    with pytest.raises(binding.SdError) as e:
+        binding.schedule_power_compute(32, 32, 4, 0, 65536, 8)
+    assert e.value.code == binding.SD_ERR_ARG
+    # well inside the limit the table is still the oracle's
+    assert binding.schedule_power_compute(32, 32, 4, 0, 4097, 8) == tuple(O.schedule_power(32, 4, 0, 4097, 32, 8))
+    assert binding.schedule_power_compute(32, 32, 4, 0, 65536, 4) == tuple(O.schedule_power(32, 4, 0, 65536, 32, 4))

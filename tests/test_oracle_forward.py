@@ -373,3 +373,22 @@ def test_ragged_budget_goes_by_slot_not_by_row_position():
     # the shifted row really differs from running it with the unshifted table
     unshifted = O.forward_sequence(w, shape.n_heads, tokens[1:2, 3:], active[:P + G - 3], F64)[0]
     assert float((unshifted - alone).abs().max()) > 1e-6
+
+
+def test_greedy_takes_the_lowest_index_of_the_maximum():
+    # the decoding rule of the five configurations: argmax, exact ties to the lowest token id
+    assert O.greedy(torch.tensor([[1.0, 3.0, 3.0, 2.0]])).tolist() == [1]
+    assert O.greedy(torch.zeros(2, 9)).tolist() == [0, 0]                       # every entry ties
+    assert O.greedy(torch.tensor([[5.0, 1.0, 5.0], [0.0, 1.0, 2.0], [2.0, 1.0, 0.0]])).tolist() == [0, 2, 0]
+    x = torch.full((1, 50272), -1.0, dtype=torch.float64)
+    x[0, 50271] = x[0, 777] = 4.0
+    assert O.greedy(x).tolist() == [777]
+    x[0, 50271] = 4.0 + 1e-12                                                   # no longer a tie
+    assert O.greedy(x).tolist() == [50271]
+    assert O.greedy(torch.tensor([[-float("inf"), -3.0, -3.0]])).tolist() == [1]
+    assert O.greedy(x).dtype == torch.int32
+    # against a scan written out by hand
+    g = torch.Generator().manual_seed(3)
+    r = torch.randint(0, 4, (6, 40), generator=g).double()                      # many exact ties
+    want = [min(range(40), key=lambda i: (-float(row[i]), i)) for row in r]
+    assert O.greedy(r).tolist() == want

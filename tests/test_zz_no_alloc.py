@@ -4,7 +4,9 @@ Some users of this library run where cudaMalloc is off limits: inside a host app
 that owns all device memory, or in a serving loop that must not allocate after start-up.  For them the library offers one entry point whose only scratch
 (the split-KV attention partials) sits in an array inside the library image.  This test
 calls it through the C ABI on two consecutive decode steps and checks each against
-sd_decode_step on the same inputs, with the tolerance of the other parity tests.
+sd_decode_step on the same inputs (the two run the same kernels, so they may differ only by the
+order in which split sums arrive: 2e-3 in bf16 storage, 1e-5 in fp32) and against the CPU oracle
+with the tolerance of the other parity tests.
 
 It is collected last on purpose: if it fails, a run that stops at the first failure has
 already exercised everything else.  It builds all of its own state, so it passes alone
@@ -30,6 +32,8 @@ def test_static_scratch_step_matches_regular_step_twice_in_a_row(name, shape):
     dec = harness.make_decoder(wl, w)
     dec.set_option(binding.SD_OPT_ATTN_CHUNK, 32)          # several splits per (row, head): the scratch is really used
     tol = harness.TOL[name]
+    same = {"fp32": 1e-5, "bf16": 2e-3}[name]               # one GPU path against the other
+    ref = harness.oracle_run_forced(wl, w, prompts, forced)    # [B, 1 + gen_len, vocab], index 0 = prompt pass
     with torch.cuda.stream(dec.stream):
         dec.schedule(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len)
         dec.prefill(prompts)
@@ -43,7 +47,9 @@ def test_static_scratch_step_matches_regular_step_twice_in_a_row(name, shape):
             dec.decode_step_static(ids[g], wl.prompt_len + g, out)
             dec.synchronize()
             err = float((out - regular[g]).abs().max())
-            assert err <= tol, (g, err)
+            assert err <= same, (g, err)
+            err_oracle = float((out.cpu().double() - ref[:, g + 1].double()).abs().max())
+            assert err_oracle <= tol, (g, err_oracle)
             assert float(regular[g].abs().max()) > 0.05     # not a comparison of zeros
         # the two entry points may be mixed inside one sequence
         third = dec.decode_step(f[:, 2].contiguous(), wl.prompt_len + 2)
@@ -52,7 +58,8 @@ def test_static_scratch_step_matches_regular_step_twice_in_a_row(name, shape):
             dec.decode_step_static(ids[g], wl.prompt_len + g, out)
         again = dec.decode_step_static(f[:, 2].contiguous(), wl.prompt_len + 2)
         dec.synchronize()
-        assert float((again - third).abs().max()) <= tol
+        assert float((again - third).abs().max()) <= same
+        assert float((again.cpu().double() - ref[:, 3].double()).abs().max()) <= tol
     assert dec.status() == 0
     dec.close()
 
