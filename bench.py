@@ -208,27 +208,16 @@ def bench_config(wl, args):
 
 # --------------------------------------------------------------------------- GPU arm
 
-def gpu_arm(args, wl, rank, world):
+def measure_workload(name, wl, weights, args, device, dist, world, steps, warmup, e2e_steps, profile_every, full_steps):
+    """Times one workload on this rank's GPU.  Returns a dict of raw results (times are the max over ranks)."""
     from paper_2307_02628_b200 import binding
-    local = int(os.environ.get("LOCAL_RANK", 0))
-    device = torch.device(f"cuda:{local}")
-    torch.cuda.set_device(device)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_
-        dist_.init_process_group("nccl", device_id=device)
-        dist = dist_
     s, B, P, G = wl.shape, wl.batch, wl.prompt_len, wl.gen_len
-    t0 = time.perf_counter()
-    weights = synth.make_weights(s, seed=0, threads=torch.get_num_threads())
-    t_weights = time.perf_counter() - t0
-
     free, _total = torch.cuda.mem_get_info(device)
     wbytes = sum(t.numel() * t.element_size() for t in [weights["tok_emb"], weights["pos_emb"]] +
                  [t for lw in weights["layers"] for t in lw.values()])
     cfg = binding.make_config(s, B, P, G)
     need_full = binding.arena_bytes(cfg, binding.SdPlan(wl.max_layers, wl.min_layers, wl.warmup, G, 1))
-    full_ok = (not args.no_full_layer) and need_full + wbytes + (4 << 30) < free
+    full_ok = full_steps > 0 and need_full + wbytes + (4 << 30) < free
     dec = binding.Decoder(s, weights, B, P, G, plan=(wl.max_layers, wl.min_layers, wl.warmup, G),
                           full_capacity=full_ok, device=str(device))
     stream = dec.stream
@@ -295,34 +284,34 @@ def gpu_arm(args, wl, rank, world):
         stream.synchronize()
         t_prefill = time.perf_counter() - tp0
 
-        for _ in range(args.warmup):
+        for _ in range(warmup):
             one_pass()
         clocks = ClockSampler(device)
         clocks.start()
         l0 = dec.launch_count()
-        ms_step = timed(one_pass, args.steps)
+        ms_step = timed(one_pass, steps)
         launches = dec.launch_count() - l0
         clock_info = clocks.stop()
         assert dec.status() == 0, "device status word set"
 
         # end to end: host ids in, logits out, every step, through sd_decode_step_host
-        h_ids = forced.t().contiguous().pin_memory()            # [G, B]
-        h_logits = torch.empty(B, s.vocab, dtype=torch.float32).pin_memory()
-
-        def e2e_pass():
-            dec.rewind()
-            for g in range(G_run):
-                dec.decode_step_host(h_ids[g], P + g, h_logits)
-
         e2e_s = float("nan")
-        if args.e2e_steps > 0:
+        if e2e_steps > 0:
+            h_ids = forced.t().contiguous().pin_memory()            # [G, B]
+            h_logits = torch.empty(B, s.vocab, dtype=torch.float32).pin_memory()
+
+            def e2e_pass():
+                dec.rewind()
+                for g in range(G_run):
+                    dec.decode_step_host(h_ids[g], P + g, h_logits)
+
             e2e_pass()
             barrier()
             te = time.perf_counter()
-            for _ in range(args.e2e_steps):
+            for _ in range(e2e_steps):
                 e2e_pass()
             barrier()
-            e2e_s = (time.perf_counter() - te) / args.e2e_steps
+            e2e_s = (time.perf_counter() - te) / e2e_steps
         e2e_s = max_over_ranks(e2e_s, dist, device)
 
         # dominant kernel (decode attention): device time per launch on sampled steps
@@ -331,8 +320,8 @@ def gpu_arm(args, wl, rank, world):
         dec.greedy(logits0, ids)
         attn_bytes = 0.0
         e = 4 if s.dtype == "fp32" else 2
-        for g in range(G_run if args.profile_every > 0 else 0):
-            sampled = (g % args.profile_every == 0)
+        for g in range(G_run if profile_every > 0 else 0):
+            sampled = (g % profile_every == 0)
             dec.set_option(binding.SD_OPT_TIMING, 1 if sampled else 0)
             dec.decode_step(ids, P + g, logits)
             dec.greedy(logits, ids)
@@ -340,17 +329,16 @@ def gpu_arm(args, wl, rank, world):
                 attn_bytes += n_active[g] * 2.0 * (P + g + 1) * s.d_model * B * e
         dec.set_option(binding.SD_OPT_TIMING, 0)
         kt = dec.kernel_times()
-        attn_ms, attn_n = kt["attention"]
 
         full = None
         if full_ok:
             dec.schedule(s.n_layers, s.n_layers, 0, G)
             one_pass()
-            ms_full = timed(one_pass, max(1, min(2, args.steps)))
+            ms_full = timed(one_pass, full_steps)
             full = {"ms_per_step": ms_full, "tokens_per_s": world * B * G_run / (ms_full / 1e3),
                     "speedup_skip_over_full": ms_full / ms_step,
                     "byte_model_bound": step_bytes(wl, [s.n_layers] * G_run) / step_bytes(wl, n_active[:G_run])}
-        elif not args.no_full_layer and G_run == G:
+        elif full_steps > 0 and G_run == G:
             # The all-layers cache for the whole generation does not fit beside the weights (config 5:
             # 172 GB): compare over the longest prefix of positions whose full cache does fit, skip and
             # full-layer both timed on exactly those positions.
@@ -364,7 +352,7 @@ def gpu_arm(args, wl, rank, world):
                     break
             if Gp:
                 one_pass(Gp)
-                ms_skip_p = timed(lambda: one_pass(Gp), max(1, min(2, args.steps)))
+                ms_skip_p = timed(lambda: one_pass(Gp), full_steps)
                 dec.close()
                 torch.cuda.empty_cache()
                 dec2 = binding.Decoder(s, weights, B, P, Gp, plan=(s.n_layers, s.n_layers, 0, Gp), full_capacity=True,
@@ -372,46 +360,97 @@ def gpu_arm(args, wl, rank, world):
                 dec2.schedule(s.n_layers, s.n_layers, 0, Gp)
                 dec2.prefill(prompts, logits0)
                 one_pass(Gp, dec2)
-                ms_full_p = timed(lambda: one_pass(Gp, dec2), max(1, min(2, args.steps)))
+                ms_full_p = timed(lambda: one_pass(Gp, dec2), full_steps)
                 assert dec2.status() == 0
                 dec2.close()
                 full = {"prefix_steps": Gp, "ms_full": ms_full_p, "ms_skip_same_steps": ms_skip_p,
                         "speedup_skip_over_full": ms_full_p / ms_skip_p,
                         "byte_model_bound": step_bytes(wl, [s.n_layers] * Gp) / step_bytes(wl, n_active[:Gp]),
                         "note": f"all-layers cache for all {G} steps does not fit; both timed on the first {Gp} positions"}
+    dec.close()
+    torch.cuda.empty_cache()
+    return {"name": name, "wl": wl, "G_run": G_run, "n_active": n_active, "ms_step": ms_step, "launches": launches,
+            "clocks": clock_info, "e2e_s": e2e_s, "attn_bytes": attn_bytes, "kt": kt, "full": full, "prefill_s": t_prefill}
 
+
+def roofline_entry(r, peak, peak_kind):
+    """The dominant kernel's roofline object from a measure_workload result."""
+    s = r["wl"].shape
+    attn_ms, attn_n = r["kt"]["attention"]
+    achieved = r["attn_bytes"] / (attn_ms / 1e3) / 1e9 if attn_ms > 0 else None
+    same_kernel = attention_kernel_hash() == ATTN_KERNEL_SHA256 and s.dtype == "bf16"
+    return {"kernel": "attn_partial_kernel (split-KV decode attention)", "bound": "hbm", "achieved": achieved,
+            "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
+            "traffic": (ATTN_TRAFFIC_RATIO * r["attn_bytes"] / attn_n if attn_n and same_kernel else None),
+            "traffic_source": ("ncu capture of this kernel source on a 2-layer case of the same launch shape, scaled by the keys read"
+                               if attn_n and same_kernel else None),
+            "launches_timed": int(attn_n),
+            "algorithmic_bytes_per_launch": r["attn_bytes"] / attn_n if attn_n else None}
+
+
+def gpu_arm(args, wl, rank, world):
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    device = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist_.init_process_group("nccl", device_id=device)
+        dist = dist_
+    s, B = wl.shape, wl.batch
+    t0 = time.perf_counter()
+    weights = synth.make_weights(s, seed=0, threads=torch.get_num_threads())
+    t_weights = time.perf_counter() - t0
+
+    r = measure_workload(args.config, wl, weights, args, device, dist, world, args.steps, args.warmup, args.e2e_steps,
+                         args.profile_every, 0 if args.no_full_layer else max(1, min(2, args.steps)))
     peak, peak_kind = measured_peaks()
+    G_run, n_active, ms_step = r["G_run"], r["n_active"], r["ms_step"]
     value = job_tokens_per_s(world, B, G_run, ms_step)
     total_bytes = step_bytes(wl, n_active[:G_run])
-    achieved = attn_bytes / (attn_ms / 1e3) / 1e9 if attn_ms > 0 else None
+    kt = r["kt"]
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic", "config": bench_config(wl, args),
-        "clocks": clock_info, "gpu_launches": int(launches),
-        "e2e": {"value": world * B * G_run / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": G_run * B * 4,
+        "clocks": r["clocks"], "gpu_launches": int(r["launches"]),
+        "e2e": {"value": world * B * G_run / r["e2e_s"], "unit": "tokens/s", "h2d_bytes_per_step": G_run * B * 4,
                 "d2h_bytes_per_step": G_run * B * s.vocab * 4},
-        "roofline": {"kernel": "attn_partial_kernel (split-KV decode attention)", "bound": "hbm", "achieved": achieved,
-                     "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
-                     "traffic": (ATTN_TRAFFIC_RATIO * attn_bytes / attn_n
-                                 if attn_n and attention_kernel_hash() == ATTN_KERNEL_SHA256 and s.dtype == "bf16" else None),
-                     "launches_timed": int(attn_n),
-                     "algorithmic_bytes_per_launch": attn_bytes / attn_n if attn_n else None},
+        "roofline": roofline_entry(r, peak, peak_kind),
         "step_roofline": {"algorithmic_bytes_per_step": total_bytes, "achieved_gbs": total_bytes / (ms_step / 1e3) / 1e9,
                           "frac_of_measured_hbm": total_bytes / (ms_step / 1e3) / 1e9 / peak,
                           "frac_of_8tbs": total_bytes / (ms_step / 1e3) / 1e9 / 8000.0},
         "kernel_time_ms": {k: v[0] for k, v in kt.items()}, "kernel_launches_timed": {k: v[1] for k, v in kt.items()},
-        "full_layer": full, "prefill_s": t_prefill, "weights_s": t_weights,
+        "full_layer": r["full"], "prefill_s": r["prefill_s"], "weights_s": t_weights,
         "mean_active_layers": sum(n_active) / len(n_active),
     }
-    if G_run != G:
-        line["partial_pass"] = f"first {G_run} of {G} decode steps per pass: a profiler run, not a benchmark value"
-    dec.close()
+    if G_run != wl.gen_len:
+        line["partial_pass"] = f"first {G_run} of {wl.gen_len} decode steps per pass: a profiler run, not a benchmark value"
+
+    # The other configurations that are large enough to time (the 1.3B shape and the batch-256 case), in short:
+    # one warm-up pass and two timed passes each, same kernels, same clock rules.  Config 5 shares config 4's weights.
+    if args.config == "c4" and world == 1 and not args.no_other_configs and args.max_gen_steps <= 0:
+        others = {}
+        for name in ("c3", "c5"):
+            wl2 = synth.CONFIGS[name]
+            w2 = weights if wl2.shape == s else synth.make_weights(wl2.shape, seed=0, threads=torch.get_num_threads())
+            r2 = measure_workload(name, wl2, w2, args, device, dist, world, 2, 1, 0, args.profile_every, 1)
+            b2 = step_bytes(wl2, r2["n_active"])
+            rf = roofline_entry(r2, peak, peak_kind)
+            others[name] = {"workload": bench_config(wl2, args)["workload"].replace(args.config + ":", name + ":", 1),
+                            "value": job_tokens_per_s(world, wl2.batch, wl2.gen_len, r2["ms_step"]), "unit": "tokens/s",
+                            "ms_per_step": r2["ms_step"], "steps": 2, "warmup": 1, "clocks": r2["clocks"],
+                            "step_roofline_frac_of_measured_hbm": b2 / (r2["ms_step"] / 1e3) / 1e9 / peak,
+                            "attention_gbs": rf["achieved"], "attention_frac": rf["frac"], "full_layer": r2["full"],
+                            "prefill_s": r2["prefill_s"]}
+            del w2
+        line["other_configs"] = others
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = torch.get_num_threads()
         tps, sec = oracle_sample(wl, weights, args.ref_rows, args.ref_steps, 2, 1)
         line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                                "sample": f"{args.ref_rows} batch row(s), 2 timed calls of {args.ref_steps} decode step(s) from position {P}, fp32, after an untimed prompt pass"}
+                                "sample": f"{args.ref_rows} batch row(s), 2 timed calls of {args.ref_steps} decode step(s) from position {wl.prompt_len}, fp32, after an untimed prompt pass"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
@@ -439,6 +478,7 @@ def main():
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")
     ap.add_argument("--no-full-layer", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="with the default workload (c4): do not also time c3 and c5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-rows", type=int, default=1)
     ap.add_argument("--ref-steps", type=int, default=1)

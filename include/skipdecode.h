@@ -147,6 +147,7 @@ int sd_layer_capacity(const sd_config *cfg, const sd_plan *plan, int32_t *capaci
 
 /* Processes the prompt with all layers (Section 2.3): fills cache positions
  * 0..P-1 of every layer and writes the logits of position P-1.
+ * The device status word is cleared (on the stream) before the work.
  * d_tokens: device int32 [B, P] row-major, ids in [0, vocab).  d_logits: device
  * fp32 [B, vocab].  1 <= B <= max_batch, 1 <= P <= max_prompt, P + gen_len <= max_pos.
  * Errors: SD_ERR_ARG, SD_ERR_STATE (no schedule), SD_ERR_CAPACITY, SD_ERR_CUDA. */
@@ -266,11 +267,21 @@ enum {
                               epilogue overlapped with the next tile's main loop; token tiles of 128, or of 96
                               where that takes fewer rounds of tiles per block); 2: the same with 128-token
                               tiles only; 0: one block per tile */
-  SD_OPT_GEMM_SPLITK = 11  /* 0..8, default 8 = the most splits of K for a QKV, fc1 or LM-head product whose output
+  SD_OPT_GEMM_SPLITK = 11, /* 0..8, default 8 = the most splits of K for a QKV, fc1 or LM-head product whose output
                               tiles cover fewer than half of the SMs (every split keeps at least 8 k-blocks of 64);
                               the partial tiles are parked in the arena and the block that arrives last adds them in
                               split order and runs the epilogue (results do not depend on arrival order);
                               0: K is split for the two residual products only */
+  SD_OPT_DETERMINISTIC = 12, /* 0 (default): the out-projection and fc2, whose K is split over several blocks, add their
+                              partial sums to the residual stream with atomic adds, i.e. in arrival order, so two runs
+                              can differ in the last bits; 1: these products park their partial tiles like the others and
+                              the block that arrives last adds them in split order: every run gives the same bits
+                              (measured cost: see the design doc) */
+  SD_OPT_TEST_WAIT_EXPIRY = 13 /* test hook, one shot: the next tensor-core product never reports its accumulator
+                              complete, its epilogue gives up the bounded wait after about a millisecond, writes
+                              nothing, and sets the wait-expired bit of the status word (sd_status then returns
+                              SD_ERR_DEVICE).  Nothing is left in flight and the handle stays usable: the following
+                              sd_prefill clears the status word.  The step that contained the product returns garbage. */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff

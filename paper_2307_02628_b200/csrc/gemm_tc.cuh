@@ -47,13 +47,14 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait expired).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long limit = kWaitLimit) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimit) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       atomicOr(status, STATUS_WAIT_EXPIRED);
       return false;
@@ -124,6 +125,10 @@ struct QkvOut {
   // ws_count[tile]; the block that arrives last adds the partials in split order and runs the epilogue.
   float* ws;
   int* ws_count;     // zero between launches (the last block puts it back)
+  int fix_residual;  // 1: the residual epilogue takes the same route (partials added in split order, one plain update per
+                     //    element) instead of atomic adds in arrival order: bit-identical results from run to run
+  int test_expire;   // test hook: the MMA warp never reports the accumulator complete and the epilogue gives up its wait
+                     //    after about a millisecond; every copy has landed and every MMA has been issued by then
 };
 
 // Tile-packed weights: [ceil(N/128)][K/64] tiles of 128 rows x 64 columns, each tile stored as
@@ -251,7 +256,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
         umma_commit(empty0 + 8 * s);              // the stage is free once these MMAs have read it
       }
-      if (ok) umma_commit(accum_bar);             // the accumulator is complete
+      if (ok && !qo.test_expire) umma_commit(accum_bar);   // the accumulator is complete
     }
   } else {
     pdl_wait();                                   // bias aside, the epilogue reads and writes buffers earlier kernels own
@@ -276,14 +281,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         kv_base = n < 2 * qo.d ? qo.Kc : qo.Vc;
       }
     }
-    const bool accum_ok = mbar_wait(accum_bar, 0, abort_flag, status);
+    const bool accum_ok = mbar_wait(accum_bar, 0, abort_flag, status, qo.test_expire ? 2000000LL : kWaitLimit);
     // The main loop is over: let the next kernel of the stream become resident now, so that its
     // launch and set-up overlap this kernel's epilogue (earlier would only park its blocks on the
     // SMs for the whole main loop).
     pdl_launch_dependents();
     // K split under a non-linear epilogue: park the partial tile, count arrivals, and let
     // the block that arrives last finish the tile from the parked partials
-    const bool fix = EPI != EPI_RESIDUAL_F32 && gridDim.z > 1;
+    const bool fix = (EPI != EPI_RESIDUAL_F32 || qo.fix_residual) && gridDim.z > 1;
     bool go = accum_ok;
     if (fix) {
       // the fix-up meets at a named barrier: all epilogue threads take it or none (a bounded wait may
@@ -295,7 +300,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
     if (go) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const float b = (bias != nullptr && n < N && (EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
+      // the bias goes in once: with the fix-up by the block that finishes the tile, else by the first split
+      const float b = (bias != nullptr && n < N && (fix || EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
       const int c_begin = ((warp - 2) >> 2) * GROUP_COLS;
       const int splits = (int)gridDim.z, tile_id = (int)(blockIdx.y * gridDim.x + blockIdx.x);
       float* ws_tile = fix ? qo.ws + (size_t)tile_id * splits * (NB * BM) + quarter * 32 + lane : nullptr;
@@ -364,6 +370,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               }
               else if (EPI == EPI_RELU_T)      // the result is the next product's operand: row of 2N bf16, hi | lo
                 Operand<__nv_bfloat16>::store(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)m * ldo, N, n, fmaxf(v, 0.f));
+              else if (fix) reinterpret_cast<float*>(out)[idx] += v;      // the only block that touches this tile's elements now
               else atomicAdd(reinterpret_cast<float*>(out) + idx, v);
             }
           }
@@ -411,6 +418,8 @@ struct TcContext {
   float* splitk_ws = nullptr;
   int* splitk_count = nullptr;
   int splitk = 8;        // most splits of K under a non-linear epilogue; 0: K is split for the residual products only
+  int deterministic = 0; // 1: split-K partial sums of the residual products are added in split order too (no atomics)
+  int test_expire = 0;   // test hook: the next product makes its accumulator wait expire (one shot)
   // (pointer, rows, cols, box rows) -> tensor map of a row-major bf16 matrix, 64-column boxes, 128-byte swizzle
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
 };
@@ -505,6 +514,12 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   if (epi == EPI_RESIDUAL_F32) {                 // partial sums may be added in any order
     const int tiles = ((N + tc::BM - 1) / tc::BM) * ((M + nb - 1) / nb);
     splits = std::max(1, std::min(kb_total / 4, c.sm_count / tiles));     // one wave: never more blocks than SMs
+    if (c.deterministic && c.splitk_ws) {        // ... or in split order, through the parked partial tiles
+      splits = std::max(1, std::min(splits, kSplitSlots / tiles));
+      qo.ws = c.splitk_ws;
+      qo.ws_count = c.splitk_count;
+      qo.fix_residual = 1;
+    }
   } else if (c.splitk && c.splitk_ws) {
     // The other epilogues are not linear, so the block that arrives last finishes the tile from parked
     // partials.  That costs a second pass over the tile: only where fewer than half of the SMs would hold
@@ -518,6 +533,7 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   }
   int kb_per_split = (kb_total + splits - 1) / splits;
   splits = (kb_total + kb_per_split - 1) / kb_per_split;      // no empty split
+  if (c.test_expire) { qo.test_expire = 1; c.test_expire = 0; }
   switch (nb) {
     case 16: return tc_launch<16>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);
     case 32: return tc_launch<32>(c.pdl, st, mw, mx, bias, out, ldo, M, N, K, kb_per_split, splits, epi, status, qo);

@@ -488,7 +488,7 @@ int decode_step_impl(sd_handle* h, const int32_t* d_ids, int position, float* d_
   const bool bf = h->cfg.dtype == SD_DTYPE_BF16;
   int err = 0;
   int64_t launched = 0;
-  const bool graphs = h->opt_graphs && !h->opt_timing && h->stream != nullptr;
+  const bool graphs = h->opt_graphs && !h->opt_timing && !h->tc.test_expire && h->stream != nullptr;
   if (!graphs) {
     err = bf ? enqueue_decode<bf16>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0, &launched)
              : enqueue_decode<float>(h, d_ids, position, false, d_logits, n, chunk, n_chunks, h->opt_timing != 0, &launched);
@@ -703,6 +703,8 @@ int sd_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_log
       if (h->pad[b] >= P) return SD_ERR_ARG;
   }
   if (h->have_rows) { h->have_rows = false; h->rows.clear(); drop_graphs(h); }   // a new batch: all rows generate
+  // a new batch starts with a clean status word (a bit set earlier has been reported through sd_status by now or is lost)
+  if (cudaMemsetAsync(h->status(), 0, sizeof(int), h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
   const int err = h->cfg.dtype == SD_DTYPE_BF16 ? run_prefill<bf16>(h, d_tokens, B, P, d_logits)
                                                 : run_prefill<float>(h, d_tokens, B, P, d_logits);
   if (err) return err;
@@ -887,6 +889,12 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value < 0 || value >= (1 << SD_K_COUNT)) return SD_ERR_ARG;
       if (value != h->opt_pdl) drop_graphs(h);
       h->opt_pdl = value; return SD_OK;
+    case SD_OPT_DETERMINISTIC:
+      if ((value != 0) != (h->tc.deterministic != 0)) drop_graphs(h);
+      h->tc.deterministic = value ? 1 : 0; return SD_OK;
+    case SD_OPT_TEST_WAIT_EXPIRY:
+      drop_graphs(h);                       // the marked launch must not be replayed from a graph
+      h->tc.test_expire = value ? 1 : 0; return SD_OK;
     case SD_OPT_TIMING:
       if (h->opt_timing && !value) collect_timing(h);
       h->opt_timing = value ? 1 : 0; return SD_OK;

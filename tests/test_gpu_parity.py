@@ -379,3 +379,50 @@ def test_prompt_shorter_than_the_configured_maximum(dtype, max_prompt, P, B):
         assert e.value.code == binding.SD_ERR_CAPACITY
     dec.close()
     _check(gpu, ref, dtype, f"max_prompt={max_prompt} P={P} B={B} {dtype}")
+
+
+@pytest.mark.parametrize("B", [5, 40])
+def test_deterministic_option_gives_the_same_bits_every_run(B):
+    """bf16 storage splits K of the out-projection and fc2 over several blocks.  By default their partial sums reach
+    the residual stream by atomic adds (arrival order); with SD_OPT_DETERMINISTIC they are added in split order."""
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("det-bf16", 3, 1024, 8, 2048, 640, 96, "bf16")      # 16 and 32 k-blocks: K is split 4 ways
+    wl = synth.Workload(shape, B, 19, 8, 3, 2, 0)
+    w = synth.make_weights(shape, seed=23, random_ln=True)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced)
+    runs = []
+    for det, graphs in ((1, 1), (1, 1), (1, 0), (0, 1)):
+        dec = harness.make_decoder(wl, w)
+        dec.set_option(binding.SD_OPT_DETERMINISTIC, det)
+        dec.set_option(binding.SD_OPT_GRAPHS, graphs)
+        runs.append(harness.gpu_run_forced(dec, wl, prompts, forced))
+        dec.close()
+        _check(runs[-1], ref, "bf16", f"deterministic={det} graphs={graphs} B={B}")
+    assert torch.equal(runs[0], runs[1]) and torch.equal(runs[0], runs[2])
+    assert float((runs[0] - runs[3]).abs().max()) <= 2e-3
+
+
+def test_expired_device_wait_is_reported_and_the_handle_stays_usable():
+    """The bounded waits inside the tensor-core kernels: a product whose accumulator never completes (test hook) gives
+    up after about a millisecond, sets the status word, and leaves nothing in flight; sd_status reports it, and after
+    the next sd_prefill the handle computes correct results again."""
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("expiry-bf16", 2, 256, 2, 512, 640, 96, "bf16")
+    wl = synth.Workload(shape, 6, 17, 4, 2, 1, 0)
+    w = synth.make_weights(shape, seed=24)
+    prompts, forced = synth.make_prompts(wl), synth.make_forced_tokens(wl)
+    ref = harness.oracle_run_forced(wl, w, prompts, forced)
+    dec = harness.make_decoder(wl, w)
+    good = harness.gpu_run_forced(dec, wl, prompts, forced)
+    with torch.cuda.stream(dec.stream):
+        dec.rewind()
+        dec.set_option(binding.SD_OPT_TEST_WAIT_EXPIRY, 1)
+        dec.decode_step(forced[:, 0].contiguous(), wl.prompt_len)       # its first product gives up its wait
+        code = binding.lib().sd_status(dec.h, None)
+        assert code == binding.SD_ERR_DEVICE
+        assert dec.status() & 2                                         # STATUS_WAIT_EXPIRED
+    again = harness.gpu_run_forced(dec, wl, prompts, forced)            # schedule + prefill (clears the word) + all steps
+    dec.close()
+    _check(again, ref, "bf16", "after an expired wait")
+    assert float((again - good).abs().max()) <= 2e-3
