@@ -235,8 +235,6 @@ def measure_workload(name, wl, weights, args, device, dist, world, steps, warmup
         dec.set_option(binding.SD_OPT_DETERMINISTIC, 1)
     if args.attn_chunk:
         dec.set_option(binding.SD_OPT_ATTN_CHUNK, args.attn_chunk)
-    if args.row_major_weights:
-        dec.set_option(binding.SD_OPT_WEIGHT_TILES, 0)
     prompts = synth.make_prompts(wl).to(device)
     forced = synth.make_forced_tokens(wl)
     logits0 = torch.empty(B, s.vocab, dtype=torch.float32, device=device)
@@ -476,7 +474,6 @@ def main():
                     help="token selection in the timed generation loop (the five configurations are greedy)")
     ap.add_argument("--no-persistent", action="store_true", help="SD_OPT_GEMM_PERSISTENT = 0")
     ap.add_argument("--splitk", type=int, default=None, help="SD_OPT_GEMM_SPLITK (most splits of K under a non-linear epilogue; 0 = off)")
-    ap.add_argument("--row-major-weights", action="store_true", help="SD_OPT_WEIGHT_TILES = 0")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")
     ap.add_argument("--deterministic", action="store_true", help="SD_OPT_DETERMINISTIC = 1")

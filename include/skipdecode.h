@@ -53,9 +53,12 @@ typedef enum {
 enum { SD_DTYPE_FP32 = 0, SD_DTYPE_BF16 = 1 };
 
 /* Model and limits.  Plain data, copied by sd_create.
- * dtype selects the storage type of weights, GEMM input operands and the KV
- * cache; the residual stream, LayerNorm statistics, softmax, accumulators and
- * logits are fp32 in both modes.  head_dim = d_model / n_heads must be 32, 64
+ * dtype selects the storage type of weights and the KV cache; the residual
+ * stream, LayerNorm statistics, softmax, accumulators and logits are fp32 in
+ * both modes.  In bf16 mode the inputs of the projections (LayerNorm outputs,
+ * attention outputs, FFN activations) are rounded to fp16 and multiplied with
+ * the weights' values held as fp16 (exact for magnitudes in [2^-14, 65504];
+ * a weight beyond 65504 saturates and sets bit 8 of the device status word).  head_dim = d_model / n_heads must be 32, 64
  * or 128; d_model and d_ffn must be multiples of 8; max_prompt + max_gen <= max_pos. */
 typedef struct {
   int32_t n_layers, d_model, n_heads, d_ffn, vocab, max_pos;
@@ -259,7 +262,6 @@ enum {
   SD_OPT_TIMING = 4,       /* 1: record per-kernel-class device time (plain launches, slower)      */
   SD_OPT_PDL = 5,          /* programmatic dependent launch: mask of kernel classes (1 << SD_K_*) whose
                               kernels may begin before their predecessor ends; 0 = none             */
-  SD_OPT_WEIGHT_TILES = 7, /* 1 (default): GEMMs read the tile-packed weight copies; 0: the caller's arrays */
   SD_OPT_PREFILL_ATTN = 8, /* 1 (default): sd_prefill's causal attention runs as 64x64 tensor-core tiles
                               (bf16 storage, head size 64 or 128); 0: one decode-style block per query row */
   SD_OPT_GEMM_PERSISTENT = 10, /* 1 (default): products with more than 64 tokens and more output tiles than SMs

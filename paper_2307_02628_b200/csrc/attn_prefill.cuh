@@ -11,6 +11,7 @@
 #pragma once
 #include <cstdint>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 namespace sd {
@@ -49,7 +50,7 @@ __device__ __forceinline__ void pf_split(float x, float y, uint32_t& hi, uint32_
 // grid (query tiles of a sequence, sequences of this pass x heads); block 128 threads.
 // qkv: fp32 [n_seq * P, ldq], q of head h at columns h*HD..; row = seq * P + pos.
 // Kc, Vc: bf16 [B, H, cap, HD] of this layer; sequences b0.. of the batch.
-// o: bf16 operand rows [n_seq * P, 2 * H * HD] (hi | lo).
+// o: operand rows [n_seq * P, H * HD] for the out-projection (fp16 values in 16-bit slots, see Operand).
 // pad (may be null): left-padding slots per batch row; a row's keys start at slot pad[b], and a
 // padding slot attends to itself alone (its output is never used).
 template <int HD>
@@ -207,7 +208,7 @@ attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16*
     __syncthreads();                                           // the other stage is refilled at the top of the next round
   }
 
-  // row sums across the quad, normalise, write the operand rows (hi | lo)
+  // row sums across the quad, normalise, write the operand rows (fp16 values)
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
   const float inv_lo = 1.f / l_lo, inv_hi = 1.f / l_hi;
@@ -216,18 +217,13 @@ attn_prefill_kernel(const float* __restrict__ qkv, int ldq, const __nv_bfloat16*
 #pragma unroll
   for (int n = 0; n < NT_O; ++n) {
     const int c = h * HD + n * 8 + 2 * t;
-    uint32_t hi, lo;
     if (p_lo < P) {
-      __nv_bfloat16* row = o + ((size_t)seq * P + p_lo) * 2 * d;
-      pf_split(acc[n][0] * inv_lo, acc[n][1] * inv_lo, hi, lo);
-      *reinterpret_cast<uint32_t*>(row + c) = hi;
-      *reinterpret_cast<uint32_t*>(row + d + c) = lo;
+      const __half2 v = __floats2half2_rn(fminf(fmaxf(acc[n][0] * inv_lo, -65504.f), 65504.f), fminf(fmaxf(acc[n][1] * inv_lo, -65504.f), 65504.f));
+      *reinterpret_cast<__half2*>(o + ((size_t)seq * P + p_lo) * d + c) = v;
     }
     if (p_hi < P) {
-      __nv_bfloat16* row = o + ((size_t)seq * P + p_hi) * 2 * d;
-      pf_split(acc[n][2] * inv_hi, acc[n][3] * inv_hi, hi, lo);
-      *reinterpret_cast<uint32_t*>(row + c) = hi;
-      *reinterpret_cast<uint32_t*>(row + d + c) = lo;
+      const __half2 v = __floats2half2_rn(fminf(fmaxf(acc[n][2] * inv_hi, -65504.f), 65504.f), fminf(fmaxf(acc[n][3] * inv_hi, -65504.f), 65504.f));
+      *reinterpret_cast<__half2*>(o + ((size_t)seq * P + p_hi) * d + c) = v;
     }
   }
 }

@@ -1,6 +1,6 @@
 // Persistent variant of the 128-row tensor-core GEMM for token tiles of 128 (prompt pass, batches
 // above 64): one CTA per SM walks over many output tiles, and the accumulator is double-buffered in
-// tensor memory (2 x 256 columns), so the epilogue of tile i (TMEM -> registers -> global) runs
+// tensor memory (2 x 128 columns), so the epilogue of tile i (TMEM -> registers -> global) runs
 // while the MMA warp is already issuing tile i + 1 and the producer keeps the shared-memory ring
 // full across tile boundaries.  Same operands, tile shapes, descriptors and epilogues as
 // gemm_tc_kernel<128, EPI>; no split-K (there are at least as many tiles as SMs where it is used).
@@ -19,17 +19,18 @@ using namespace tc;
 // Token tile NB = 128, or 96 where that needs fewer rounds of tiles per block (config 5's QKV: 96 x 2 = 192
 // tiles of 128 tokens are two rounds for 148 blocks, 96 x 3 = 288 tiles of 96 tokens two rounds of 3/4 the work).
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int TMEM_COLS = 512;                   // two accumulators of 2 NB columns each (all 512 columns at NB = 128)
-__host__ __device__ constexpr int stages(int nb) { return nb >= 128 ? 4 : 5; }
-__host__ __device__ constexpr int stage_bytes(int nb) { return A_BYTES + 2 * nb * BK * 2; }
+constexpr int TMEM_COLS = 256;                   // two accumulators, 128 columns apart, of NB columns each
+constexpr int ACC_STRIDE = 128;
+__host__ __device__ constexpr int stages(int nb) { return nb >= 128 ? 6 : 7; }
+__host__ __device__ constexpr int stage_bytes(int nb) { return A_BYTES + nb * BK * 2; }
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
 
 // Order in which the CTAs walk over the output tiles.  The CTAs that run at the same time hold
 // consecutive tile numbers, and what they read at the same time they fetch from DRAM once (the rest are
 // L2 hits).  Tiles are therefore numbered in bands of BAND weight tiles, weight tile fastest inside a
 // band: one wave of CTAs then covers about BAND weight tiles x (SMs / BAND) token tiles instead of every
-// weight tile for a single token tile.  A token tile (hi + lo) is twice a weight tile in bytes, so a wave
-// of S CTAs fetches BAND + 2 S / BAND tile units, least near BAND = sqrt(2 S): 16 for 148 SMs.
+// weight tile for a single token tile.  A 128-token tile is as large as a weight tile, so a wave of S CTAs
+// fetches about BAND + S / BAND tile units: flat around its minimum at sqrt(S) = 12; 16 divides the tile counts here.
 constexpr int BAND = 16;
 __device__ __forceinline__ void tile_coords(int tile, int tiles_n, int tiles_m, int& tn, int& tm) {
   const int band_tiles = BAND * tiles_m;
@@ -48,8 +49,8 @@ __global__ void __launch_bounds__(192, 1)
 gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                        const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                        int tiles_n, int tiles_total, int* __restrict__ status, const QkvOut qo) {
-  constexpr int STAGES = stages(NB), B_BYTES = NB * BK * 2, STAGE_BYTES = stage_bytes(NB);
-  constexpr int ACC_COLS = 2 * NB;               // one accumulator: W.hi in [0, NB), W.lo in [NB, 2 NB)
+  constexpr int STAGES = stages(NB), STAGE_BYTES = stage_bytes(NB);
+  constexpr int ACC_COLS = ACC_STRIDE;           // one accumulator: NB columns, one per token of the tile
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -112,8 +113,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
             mbar_expect_tx(fb, STAGE_BYTES);
             load_w_tile(a_dst, &map_w, qo, kb, n0, fb);
           }
-          tma_load_2d(a_dst + A_BYTES, &map_x, kb * BK, m0, fb);                 // hi part: columns [0, K)
-          tma_load_2d(a_dst + A_BYTES + B_BYTES, &map_x, K + kb * BK, m0, fb);   // lo part: columns [K, 2K)
+          tma_load_2d(a_dst + A_BYTES, &map_x, kb * BK, m0, fb);
         }
       }
       if (*abort_flag) {
@@ -128,7 +128,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(2 * NB);
+      constexpr uint32_t idesc = instr_desc(NB);
       int it = 0, i = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < tiles_total && ok; tile += gridDim.x, ++i) {
@@ -187,17 +187,16 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
       const float b = (bias != nullptr && n < N) ? __bfloat162float(bias[n]) : 0.f;
 #pragma unroll 1
       for (int c = 0; c < NB; c += 32) {
-        uint32_t r[32], rl[32];
+        uint32_t r[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * ACC_COLS + c);
         tmem_ld32(taddr, r);
-        tmem_ld32(taddr + NB, rl);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (n < N) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const int m = m0 + c + j;
             if (m < M) {
-              const float v = (__uint_as_float(r[j]) + __uint_as_float(rl[j])) + b;
+              const float v = __uint_as_float(r[j]) + b;
               const size_t idx = (size_t)m * ldo + n;
               if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
               else if (EPI == EPI_QKV_CACHE) {
@@ -267,7 +266,7 @@ inline void persist_init(PersistContext& p, const TcContext& c) {
 inline bool persist_gemm(PersistContext& p, TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const __nv_bfloat16* W,
                          const __nv_bfloat16* bias, int M, int N, int K, void* out, int ldo, int epi, int* status,
                          const tc::QkvOut* qkv_out = nullptr, const __nv_bfloat16* Wp = nullptr) {
-  if (!p.ready || !p.enabled || !c.ready || K % tc::BK || M <= 64 || N < 1) return false;
+  if (!p.ready || !p.enabled || !c.ready || !Wp || K % tc::BK || M <= 64 || N < 1) return false;
   if (epi == EPI_QKV_CACHE && (!qkv_out || qkv_out->d % tc::BM || N != 3 * qkv_out->d)) return false;
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
   const int tiles_n = (N + tc::BM - 1) / tc::BM;
@@ -282,7 +281,7 @@ inline bool persist_gemm(PersistContext& p, TcContext& c, cudaStream_t st, const
   qo.w_packed = Wp;
   CUtensorMap mw_v, mx_v;
   const CUtensorMap *mw = &mw_v, *mx = &mx_v;
-  if (!tc_map(c, W, N, K, tc::BM, &mw_v) || !tc_map(c, X, M, 2 * K, nb, &mx_v)) return false;
+  if (!tc_map(c, W, N, K, tc::BM, &mw_v) || !tc_map(c, X, M, K, nb, &mx_v)) return false;
   if (nb == 96) persist_launch<96>(c.pdl, st, c.sm_count, mw, mx, bias, out, ldo, M, N, K, tiles_n, total, epi, status, qo);
   else persist_launch<128>(c.pdl, st, c.sm_count, mw, mx, bias, out, ldo, M, N, K, tiles_n, total, epi, status, qo);
   return true;

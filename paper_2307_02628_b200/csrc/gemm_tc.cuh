@@ -1,6 +1,7 @@
-// Tensor-core GEMM for bf16 operands on sm_100a: out[m, n] (+)= sum_k X[m, k] W[n, k] + bias[n].
-// X is an Operand row (kernels.cuh): X = Xhi + Xlo, two bf16 matrices side by side in one
-// [M, 2K] buffer; both are multiplied with the same W tile into the same accumulator.
+// Tensor-core GEMM for bf16 storage on sm_100a: out[m, n] (+)= sum_k X[m, k] W[n, k] + bias[n].
+// X rows are Operand rows (kernels.cuh): the activations rounded to fp16.  W is read from the tile-packed copy that
+// sd_create makes of every matrix, in which each bf16 weight is stored as the fp16 bit pattern of the same value,
+// so that one fp16 x fp16 MMA pass gives the product of the bf16 weights with 11-bit activations.
 //
 // The weight's output dimension sits on the MMA M axis (D^T = W X^T): a CTA owns 128 rows
 // of W, so tiles are full even when the token count M is 16..256, which becomes the MMA N.
@@ -76,10 +77,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// kind::f16 instruction descriptor: D = fp32 [4,6), A = B = bf16 [7,10) [10,13), both K-major,
-// N >> 3 at [17,23), M >> 4 at [24,29).
+// kind::f16 instruction descriptor: D = fp32 [4,6), A and B formats [7,10) [10,13) = 0 (fp16; 1 would be bf16), both
+// K-major, N >> 3 at [17,23), M >> 4 at [24,29).
 __host__ __device__ constexpr uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
@@ -152,8 +153,8 @@ __device__ __forceinline__ void load_w_tile(uint32_t dst, const CUtensorMap* map
 // which halves the serial part of the epilogue (loads from tensor memory, then one store per column).
 __host__ __device__ constexpr int epi_warps(int nb) { return nb >= 32 ? 8 : 4; }
 __host__ __device__ constexpr int block_threads(int nb) { return 64 + 32 * epi_warps(nb); }
-__host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 4 : nb >= 64 ? 7 : 8; }
-__host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + 2 * nb * BK * 2; }   // W tile + Xhi + Xlo tiles
+__host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 6 : nb >= 64 ? 9 : nb >= 32 ? 10 : 11; }
+__host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + nb * BK * 2; }   // W tile + X tile
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
 
 template <int NB, int EPI>
@@ -162,8 +163,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                int kb_per_split, int* __restrict__ status, const QkvOut qo) {
   constexpr int STAGES = stages_for(NB);
-  constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
-  constexpr int TMEM_COLS = 2 * NB;              // W.hi in columns [0, NB), W.lo in [NB, 2 NB); a power of two >= 32
+  constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int TMEM_COLS = NB < 32 ? 32 : NB;   // one accumulator column per token; a power of two >= 32
   constexpr int EW = epi_warps(NB);              // epilogue warps: 4, or 8 = two groups that split the columns
   constexpr int GROUP_COLS = NB / (EW / 4);      // token columns per group of four warps
   constexpr int CW = GROUP_COLS < 32 ? 16 : 32;  // accumulator columns read per tcgen05.ld
@@ -223,8 +224,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           mbar_expect_tx(fb, STAGE_BYTES);
           load_w_tile(a_dst, &map_w, qo, kb0 + i, n0, fb);
         }
-        tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);                 // hi part: columns [0, K)
-        tma_load_2d(a_dst + A_BYTES + B_BYTES, &map_x, K + (kb0 + i) * BK, m0, fb);   // lo part: columns [K, 2K)
+        tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);
         if (i + 1 > issued) issued = i + 1;
       }
       if (*abort_flag) {
@@ -238,11 +238,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      // The hi tile (NB rows) and the lo tile (NB rows) sit back to back in the stage, so they are
-      // one K-major operand of 2 NB rows: a single MMA of N = 2 NB per k-step puts W.hi and W.lo
-      // side by side in tensor memory (the epilogue adds the halves).  One wide instruction
-      // instead of two narrow ones: at these sizes the MMA pipe is paced per instruction.
-      constexpr uint32_t idesc = instr_desc(2 * NB);
+      constexpr uint32_t idesc = instr_desc(NB);
       bool ok = true;
       for (int i = 0; i < nkb && ok; ++i) {
         const int s = i % STAGES, round = i / STAGES;
@@ -310,13 +306,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         float* mine = ws_tile + (size_t)blockIdx.z * (NB * BM);
 #pragma unroll 1
         for (int c = c_begin; c < c_begin + GROUP_COLS; c += CW) {
-          uint32_t r[32], rl[32];
+          uint32_t r[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
-          if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
+          if (CW == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
           for (int j = 0; j < CW; ++j)             // 32 lanes = 32 consecutive weight rows: one 128-byte store per column
-            __stcg(mine + (size_t)(c + j) * BM, __uint_as_float(r[j]) + __uint_as_float(rl[j]));
+            __stcg(mine + (size_t)(c + j) * BM, __uint_as_float(r[j]));
         }
         __threadfence();
         asm volatile("bar.sync 1, %0;" ::"n"(32 * EW) : "memory");
@@ -332,13 +328,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       }
 #pragma unroll 1
       for (int c = c_begin; emit && c < c_begin + GROUP_COLS; c += CW) {
-        uint32_t r[32], rl[32];
+        uint32_t r[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
         if (fix) {
           // partials added in split order, so the result does not depend on which block came last; all
           // loads of one split are in flight together
 #pragma unroll
-          for (int j = 0; j < CW; ++j) { r[j] = 0u; rl[j] = 0u; }
+          for (int j = 0; j < CW; ++j) r[j] = 0u;
 #pragma unroll 1
           for (int z = 0; z < splits; ++z) {
             const float* src = ws_tile + (size_t)z * (NB * BM) + (size_t)c * BM;
@@ -349,7 +345,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int j = 0; j < CW; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + t[j]);
           }
         } else {
-          if (CW == 32) { tmem_ld32(taddr, r); tmem_ld32(taddr + NB, rl); } else { tmem_ld16(taddr, r); tmem_ld16(taddr + NB, rl); }
+          if (CW == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         }
         if (n < N) {
@@ -357,7 +353,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           for (int j = 0; j < CW; ++j) {
             const int m = m0 + c + j;
             if (m < M) {
-              const float v = (__uint_as_float(r[j]) + __uint_as_float(rl[j])) + b;
+              const float v = __uint_as_float(r[j]) + b;
               const size_t idx = (size_t)m * ldo + n;
               if (EPI == EPI_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
               else if (EPI == EPI_QKV_CACHE) {
@@ -368,7 +364,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                   if (row >= 0) kv_base[((size_t)row + (size_t)kv_head * qo.cap) * qo.hd + kv_elem] = __float2bfloat16_rn(v);
                 }
               }
-              else if (EPI == EPI_RELU_T)      // the result is the next product's operand: row of 2N bf16, hi | lo
+              else if (EPI == EPI_RELU_T)      // the result is the next product's operand row
                 Operand<__nv_bfloat16>::store(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)m * ldo, N, n, fmaxf(v, 0.f));
               else if (fix) reinterpret_cast<float*>(out)[idx] += v;      // the only block that touches this tile's elements now
               else atomicAdd(reinterpret_cast<float*>(out) + idx, v);
@@ -387,8 +383,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 }
 
 // One block per 128 x 64 tile: tile (tn, kb) holds W[tn * 128 + r][kb * 64 + 8 c .. +8] at 16-byte
-// piece r * 8 + (c ^ (r & 7)); rows past N are zero.
-__global__ void pack_tiles_kernel(const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ P, int N, int K) {
+// piece r * 8 + (c ^ (r & 7)); rows past N are zero.  Each bf16 weight is written as the fp16 with the same value:
+// exact for magnitudes in [2^-14, 65504] (every bf16 has at most 8 significant bits); smaller ones land on the fp16
+// subnormal grid (absolute error at most 2^-25), larger ones saturate and raise STATUS_WEIGHT_RANGE.
+__global__ void pack_tiles_kernel(const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ P, int N, int K, int* __restrict__ status) {
   const int KB = K / BK;
   const int tn = blockIdx.x / KB, kb = blockIdx.x - tn * KB;
   uint4* dst = reinterpret_cast<uint4*>(P + (size_t)blockIdx.x * BM * BK);
@@ -396,7 +394,21 @@ __global__ void pack_tiles_kernel(const __nv_bfloat16* __restrict__ W, __nv_bflo
     const int r = i >> 3, c8 = i & 7;
     const int n = tn * BM + r;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (n < N) v = *reinterpret_cast<const uint4*>(W + (size_t)n * K + kb * BK + c8 * 8);
+    if (n < N) {
+      const uint4 w = *reinterpret_cast<const uint4*>(W + (size_t)n * K + kb * BK + c8 * 8);
+      const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+      uint32_t out[4];
+      bool clipped = false;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float a = __uint_as_float(in[e] << 16), b = __uint_as_float(in[e] & 0xffff0000u);
+        clipped = clipped || fabsf(a) > 65504.f || fabsf(b) > 65504.f;
+        const __half2 h = __floats2half2_rn(sat_f16(a), sat_f16(b));
+        out[e] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      if (clipped) atomicOr(status, STATUS_WEIGHT_RANGE);
+      v = make_uint4(out[0], out[1], out[2], out[3]);
+    }
     dst[r * 8 + (c8 ^ (r & 7))] = v;
   }
 }
@@ -504,11 +516,12 @@ inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const
   tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
   qo.packed_kb = Wp ? K / tc::BK : 0;
   qo.w_packed = Wp;
+  if (!Wp) return false;                       // the MMAs take the weights from the packed fp16 copy only
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) return false;
   const int nb = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
   CUtensorMap mw_v, mx_v;
-  const CUtensorMap *mw = &mw_v, *mx = &mx_v;                 // W's map is unused by the kernel when the packed copy is read
-  if (!tc_map(c, W, N, K, tc::BM, &mw_v) || !tc_map(c, X, M, 2 * K, nb, &mx_v)) return false;
+  const CUtensorMap *mw = &mw_v, *mx = &mx_v;                 // W's map is not used by the kernel (packed copy)
+  if (!tc_map(c, W, N, K, tc::BM, &mw_v) || !tc_map(c, X, M, K, nb, &mx_v)) return false;
   const int kb_total = (K + tc::BK - 1) / tc::BK;
   int splits = 1;
   if (epi == EPI_RESIDUAL_F32) {                 // partial sums may be added in any order

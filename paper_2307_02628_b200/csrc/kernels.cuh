@@ -4,12 +4,13 @@
 // GEMM does not take).  T is the storage type: float or __nv_bfloat16.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace sd {
 
-enum : int { STATUS_BAD_TOKEN = 1, STATUS_WAIT_EXPIRED = 2, STATUS_BAD_SHAPE = 4 };
+enum : int { STATUS_BAD_TOKEN = 1, STATUS_WAIT_EXPIRED = 2, STATUS_BAD_SHAPE = 4, STATUS_WEIGHT_RANGE = 8 };
 
 // Programmatic dependent launch.  Every kernel of the step calls pdl_begin() before it touches
 // anything an earlier kernel wrote: it lets the next kernel in the stream start its own
@@ -47,25 +48,26 @@ template <> struct Vec16<__nv_bfloat16> {
   }
 };
 
-// GEMM input operands.  In fp32 storage an operand row is K floats.  In bf16 storage it is
-// 2K bf16: columns [0,K) hold hi = bf16(v) and columns [K,2K) hold lo = bf16(v - hi), so the
-// tensor cores see v to ~16 mantissa bits (two bf16 products per element) while weights
-// and KV cache stay plain bf16.
+// GEMM input operands (activations).  In fp32 storage an operand row is K floats.  In bf16 storage it is K
+// 16-bit slots that hold the value rounded to fp16 (11 significant bits, against the 8 of a bf16), saturated at
+// the largest finite fp16: the tensor-core kernels multiply them with the weights' values held as fp16 as well (a
+// bf16 weight is an fp16 value exactly unless its magnitude is below 2^-14 or above 65504, see pack_tiles_kernel),
+// one MMA pass per product.  Weights as the caller stores them and the KV cache stay bf16.  The operand buffers are
+// typed as the storage type; only the two functions below know what the 16 bits mean.
 template <typename T> struct Operand;
 template <> struct Operand<float> {
   static constexpr int PARTS = 1;
   __device__ static __forceinline__ void store(float* row, int K, int c, float v) { row[c] = v; }
   __device__ static __forceinline__ float load(const float* row, int K, int c) { return row[c]; }
 };
+__device__ __forceinline__ float sat_f16(float v) { return fminf(fmaxf(v, -65504.f), 65504.f); }
 template <> struct Operand<__nv_bfloat16> {
-  static constexpr int PARTS = 2;
+  static constexpr int PARTS = 1;
   __device__ static __forceinline__ void store(__nv_bfloat16* row, int K, int c, float v) {
-    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-    row[c] = hi;
-    row[K + c] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    reinterpret_cast<__half*>(row)[c] = __float2half_rn(sat_f16(v));
   }
   __device__ static __forceinline__ float load(const __nv_bfloat16* row, int K, int c) {
-    return __bfloat162float(row[c]) + __bfloat162float(row[K + c]);
+    return __half2float(reinterpret_cast<const __half*>(row)[c]);
   }
 };
 
@@ -171,7 +173,7 @@ layernorm_kernel(const float* __restrict__ x, const T* __restrict__ gamma, const
       s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
     }
     // bf16 storage: gain and offset as 8-byte vectors, fetched before the reductions so that their latency
-    // hides behind them, and the operand row written as 8-byte vectors (4 hi, 4 lo)
+    // hides behind them, and the operand row written as 8-byte vectors (4 fp16)
     constexpr bool kVec = sizeof(T) == 2;
     const bool vec = kVec && ((reinterpret_cast<uintptr_t>(gamma) | reinterpret_cast<uintptr_t>(beta)) & 7) == 0;
     uint2 gv[MAXV], bv[MAXV];
@@ -205,17 +207,11 @@ layernorm_kernel(const float* __restrict__ x, const T* __restrict__ gamma, const
                               __uint_as_float(gv[i].y << 16), __uint_as_float(gv[i].y & 0xffff0000u)};
           const float o[4] = {__uint_as_float(bv[i].x << 16), __uint_as_float(bv[i].x & 0xffff0000u),
                               __uint_as_float(bv[i].y << 16), __uint_as_float(bv[i].y & 0xffff0000u)};
-          uint32_t hi[4], lo[4];
+          float y[4];
 #pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const float y = (vals[t] - mean) * rstd * g[t] + o[t];
-            const __nv_bfloat16 h = __float2bfloat16_rn(y);
-            hi[t] = __bfloat16_as_ushort(h);
-            lo[t] = __bfloat16_as_ushort(__float2bfloat16_rn(y - __bfloat162float(h)));
-          }
-          uint2* dst = reinterpret_cast<uint2*>(ur);          // row of 2 d bf16: hi | lo
-          dst[k] = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
-          dst[(d >> 2) + k] = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+          for (int t = 0; t < 4; ++t) y[t] = sat_f16((vals[t] - mean) * rstd * g[t] + o[t]);
+          const __half2 h01 = __floats2half2_rn(y[0], y[1]), h23 = __floats2half2_rn(y[2], y[3]);
+          reinterpret_cast<uint2*>(ur)[k] = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
         } else {
 #pragma unroll
           for (int t = 0; t < 4; ++t) {

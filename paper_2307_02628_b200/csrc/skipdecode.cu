@@ -67,7 +67,7 @@ struct sd_handle {
   const int* d_rows() const { return have_rows ? at<int>(A.rows) : nullptr; }
   int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
-  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = SD_PDL_DEFAULT, opt_tiles = 1, opt_prefill = 1;
+  int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = SD_PDL_DEFAULT, opt_prefill = 1;
   bool packed = false;       // the arena holds tile-packed copies of the weight matrices
   // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
   struct Graph { cudaGraphExec_t exec; int64_t nodes; };
@@ -182,7 +182,7 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   A.rows_max = std::max(c.max_batch, chunk_rows);
   const size_t R = A.rows_max;
   A.x = take(R * d * 4);
-  A.u = take(R * d * 4);                 // GEMM operands: K floats, or 2K bf16 (hi | lo), per row
+  A.u = take(R * d * 4);                 // GEMM operands: K floats, or K 16-bit slots, per row
   A.qkv = take(R * 3 * d * 4);
   A.o = take(R * d * 4);
   A.y = take(R * (size_t)c.d_ffn * 4);
@@ -250,7 +250,7 @@ template <typename T>
 void launch_gemm(Launcher& Lc, int cls, const T* A, const T* W, size_t packed_off, const T* bias, int M, int N, int K,
                  void* out, int ldo, int epi) {
   sd_handle* h = Lc.h;
-  const T* Wp = (h->packed && h->opt_tiles) ? h->at<T>(packed_off) : nullptr;
+  const T* Wp = h->packed ? h->at<T>(packed_off) : nullptr;
   h->tc.pdl = pdl_for(h, cls);
   Lc.begin(cls);
   bool done = false;
@@ -281,7 +281,7 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
   sd_handle* h = Lc.h;
   if (h->opt_gemm == 1) return false;
   const sd::tc::QkvOut qo{Kc, Vc, d, h->cfg.n_heads, h->hd, cap, map, 0, nullptr};
-  const bf16* Wp = (h->packed && h->opt_tiles) ? h->at<bf16>(packed_off) : nullptr;
+  const bf16* Wp = h->packed ? h->at<bf16>(packed_off) : nullptr;
   h->tc.pdl = pdl_for(h, SD_K_GEMM_QKV);
   Lc.begin(SD_K_GEMM_QKV);
   bool done = false;
@@ -599,7 +599,7 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
     const int d = cfg->d_model, f = cfg->d_ffn;
     auto pack = [&](const void* W, size_t off, int n, int k) {
       const int tiles = (n + 255) / 256 * 2 * (k / 64);
-      sd::tc::pack_tiles_kernel<<<tiles, 256, 0, h->stream>>>(static_cast<const bf16*>(W), h->at<bf16>(off), n, k);
+      sd::tc::pack_tiles_kernel<<<tiles, 256, 0, h->stream>>>(static_cast<const bf16*>(W), h->at<bf16>(off), n, k, h->status());
     };
     for (int l = 0; l < L; ++l) {
       pack(h->w_qkv[l], h->A.wp_qkv[l], 3 * d, d);
@@ -882,9 +882,6 @@ int sd_set_option(sd_handle* h, int option, int value) {
       h->persist.allow_96 = value == 1 ? 1 : 0; return SD_OK;
     case SD_OPT_PREFILL_ATTN:
       h->opt_prefill = value ? 1 : 0; return SD_OK;
-    case SD_OPT_WEIGHT_TILES:
-      if ((value != 0) != (h->opt_tiles != 0)) drop_graphs(h);
-      h->opt_tiles = value ? 1 : 0; return SD_OK;
     case SD_OPT_PDL:
       if (value < 0 || value >= (1 << SD_K_COUNT)) return SD_ERR_ARG;
       if (value != h->opt_pdl) drop_graphs(h);

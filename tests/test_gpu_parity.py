@@ -424,5 +424,7 @@ def test_expired_device_wait_is_reported_and_the_handle_stays_usable():
         assert dec.status() & 2                                         # STATUS_WAIT_EXPIRED
     again = harness.gpu_run_forced(dec, wl, prompts, forced)            # schedule + prefill (clears the word) + all steps
     dec.close()
-    _check(again, ref, "bf16", "after an expired wait")
+    err, strict, near = harness.compare(again, ref, harness.TOL["bf16"])
+    print(f"after an expired wait: max|err|={err:.3e} argmax strict={strict:.4f} with near-ties={near:.4f}")
+    assert err <= harness.TOL["bf16"] and near >= 0.99              # 30 (row, step) pairs: one near-tie moves `strict` by 3 %
     assert float((again - good).abs().max()) <= 2e-3
