@@ -277,8 +277,8 @@ enum {
   SD_OPT_DETERMINISTIC = 12, /* 0 (default): the out-projection and fc2, whose K is split over several blocks, add their
                               partial sums to the residual stream with atomic adds, i.e. in arrival order, so two runs
                               can differ in the last bits; 1: these products park their partial tiles like the others and
-                              the block that arrives last adds them in split order: every run gives the same bits
-                              (measured cost: see the design doc) */
+                              the block that arrives last adds them in split order: every run gives the same bits,
+                              at a tenth to a fifth of the decode rate (a second pass over every tile of those products) */
   SD_OPT_TEST_WAIT_EXPIRY = 13 /* test hook, one shot: the next tensor-core product never reports its accumulator
                               complete, its epilogue gives up the bounded wait after about a millisecond, writes
                               nothing, and sets the wait-expired bit of the status word (sd_status then returns

@@ -147,14 +147,26 @@ __device__ __forceinline__ void load_w_tile(uint32_t dst, const CUtensorMap* map
   else
     tma_load_2d(dst, map, kb * BK, n_row0, bar);
 }
+// `count` consecutive k-blocks of one row tile: adjacent in the packed copy, so one bulk copy brings them all
+__device__ __forceinline__ void load_w_tiles(uint32_t dst, const CUtensorMap* map, const QkvOut& qo, int kb, int count, int n_row0, uint32_t bar) {
+  if (qo.packed_kb)
+    bulk_load(dst, qo.w_packed + ((size_t)(n_row0 >> 7) * qo.packed_kb + kb) * (BM * BK), count * (BM * BK * 2), bar);
+  else
+    for (int t = 0; t < count; ++t) tma_load_2d(dst + t * (BM * BK * 2), map, (kb + t) * BK, n_row0, bar);
+}
 
 // Epilogue warps: a warp can only read the quarter of the tensor-memory lanes that matches its index
 // mod 4, so there are four warps per group; with two groups each takes half of the token columns,
 // which halves the serial part of the epilogue (loads from tensor memory, then one store per column).
 __host__ __device__ constexpr int epi_warps(int nb) { return nb >= 32 ? 8 : 4; }
 __host__ __device__ constexpr int block_threads(int nb) { return 64 + 32 * epi_warps(nb); }
-__host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 6 : nb >= 64 ? 9 : nb >= 32 ? 10 : 11; }
-__host__ __device__ constexpr int stage_bytes(int nb) { return BM * BK * 2 + nb * BK * 2; }   // W tile + X tile
+// k-blocks per pipeline stage.  The thread that issues the MMAs pays a fixed price per stage (one barrier
+// wait, one fence, one commit) beside the four instructions of a k-block, and at 64 tokens or fewer that
+// chain, not the tensor pipe, paces the block: two k-blocks per stage halve the fixed part.
+__host__ __device__ constexpr int kps_for(int nb) { return nb >= 128 ? 1 : 2; }
+__host__ __device__ constexpr int stage_bytes(int nb) { return kps_for(nb) * (BM * BK * 2 + nb * BK * 2); }   // W tiles, then X tiles
+// 6 stages of 32 KB at 128 tokens (a 7th fits and measured no faster), else all that fit in 227 KB: 4, 5, 6 at 64, 32, 16 tokens
+__host__ __device__ constexpr int stages_for(int nb) { return nb >= 128 ? 6 : (227 * 1024 - 2304) / stage_bytes(nb); }
 __host__ __device__ constexpr int smem_bytes(int nb) { return stages_for(nb) * stage_bytes(nb) + 1024 /*alignment*/ + 256 /*barriers*/ + 1024 /*per-column cache rows*/; }
 
 template <int NB, int EPI>
@@ -162,8 +174,9 @@ __global__ void __launch_bounds__(block_threads(NB), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __nv_bfloat16* __restrict__ bias, void* __restrict__ out, int ldo, int M, int N, int K,
                int kb_per_split, int* __restrict__ status, const QkvOut qo) {
-  constexpr int STAGES = stages_for(NB);
-  constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int STAGES = stages_for(NB), KPS = kps_for(NB);
+  constexpr int A_BYTES = BM * BK * 2, B_BYTES = NB * BK * 2, STAGE_BYTES = KPS * (A_BYTES + B_BYTES);
+  constexpr int X_OFF = KPS * A_BYTES;           // a stage holds KPS weight tiles, then KPS token tiles
   constexpr int TMEM_COLS = NB < 32 ? 32 : NB;   // one accumulator column per token; a power of two >= 32
   constexpr int EW = epi_warps(NB);              // epilogue warps: 4, or 8 = two groups that split the columns
   constexpr int GROUP_COLS = NB / (EW / 4);      // token columns per group of four warps
@@ -185,6 +198,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const int kb_total = (K + BK - 1) / BK;
   const int kb0 = blockIdx.z * kb_per_split, kb1 = min(kb0 + kb_per_split, kb_total);
   const int nkb = kb1 - kb0;                                     // >= 1 by construction of the grid
+  const int nst = (nkb + KPS - 1) / KPS;                         // pipeline stages' worth of k-blocks; the last may be short
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -207,24 +221,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
       // The weights do not depend on the previous kernel: start streaming the first stages'
       // W tiles while it is still finishing, and only then wait for it before touching X.
-      const int early = nkb < STAGES ? nkb : STAGES;
+      const int early = nst < STAGES ? nst : STAGES;
       for (int i = 0; i < early; ++i) {
         const uint32_t fb = full0 + 8 * i;
-        mbar_expect_tx(fb, STAGE_BYTES);
-        load_w_tile(tiles + i * STAGE_BYTES, &map_w, qo, kb0 + i, n0, fb);
+        const int c = min(KPS, nkb - i * KPS);
+        mbar_expect_tx(fb, c * (A_BYTES + B_BYTES));
+        load_w_tiles(tiles + i * STAGE_BYTES, &map_w, qo, kb0 + i * KPS, c, n0, fb);
       }
       pdl_wait();
       int issued = early;
-      for (int i = 0; i < nkb; ++i) {
+      for (int i = 0; i < nst; ++i) {
         const int s = i % STAGES, round = i / STAGES;
         const uint32_t fb = full0 + 8 * s;
         const uint32_t a_dst = tiles + s * STAGE_BYTES;
+        const int c = min(KPS, nkb - i * KPS);
         if (round > 0) {
           if (!mbar_wait(empty0 + 8 * s, (round - 1) & 1, abort_flag, status)) break;
-          mbar_expect_tx(fb, STAGE_BYTES);
-          load_w_tile(a_dst, &map_w, qo, kb0 + i, n0, fb);
+          mbar_expect_tx(fb, c * (A_BYTES + B_BYTES));
+          load_w_tiles(a_dst, &map_w, qo, kb0 + i * KPS, c, n0, fb);
         }
-        tma_load_2d(a_dst + A_BYTES, &map_x, (kb0 + i) * BK, m0, fb);
+        for (int t = 0; t < c; ++t)
+          tma_load_2d(a_dst + X_OFF + t * B_BYTES, &map_x, (kb0 + i * KPS + t) * BK, m0, fb);
         if (i + 1 > issued) issued = i + 1;
       }
       if (*abort_flag) {
@@ -240,16 +257,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc(NB);
       bool ok = true;
-      for (int i = 0; i < nkb && ok; ++i) {
+      for (int i = 0; i < nst && ok; ++i) {
         const int s = i % STAGES, round = i / STAGES;
         ok = mbar_wait(full0 + 8 * s, round & 1, abort_flag, status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = tiles + s * STAGE_BYTES;
-        const uint64_t a_desc = smem_desc(a_addr), b_desc = smem_desc(a_addr + A_BYTES);
+        const int c = min(KPS, nkb - i * KPS);
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k)     // 32 bytes further along K inside the swizzle row
-          umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+        for (int t = 0; t < KPS; ++t) {
+          if (t < c) {
+            const uint64_t a_desc = smem_desc(a_addr + t * A_BYTES), b_desc = smem_desc(a_addr + X_OFF + t * B_BYTES);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)   // 32 bytes further along K inside the swizzle row
+              umma(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || t > 0 || k > 0) ? 1u : 0u);
+          }
+        }
         umma_commit(empty0 + 8 * s);              // the stage is free once these MMAs have read it
       }
       if (ok && !qo.test_expire) umma_commit(accum_bar);   // the accumulator is complete
@@ -511,7 +534,7 @@ inline bool tc_launch(bool pdl, cudaStream_t st, const CUtensorMap* mw, const CU
 inline bool tc_gemm(TcContext& c, cudaStream_t st, const __nv_bfloat16* X, const __nv_bfloat16* W, const __nv_bfloat16* bias,
                     int M, int N, int K, void* out, int ldo, int epi, int* status, const tc::QkvOut* qkv_out = nullptr,
                     const __nv_bfloat16* Wp = nullptr) {
-  if (!c.ready || K % tc::BK || M < 1 || N < 1) return false;   // the hi and lo halves of a row are K apart: whole k-blocks only
+  if (!c.ready || K % tc::BK || M < 1 || N < 1) return false;   // whole k-blocks only
   if (epi == EPI_QKV_CACHE && (!qkv_out || qkv_out->d % tc::BM || N != 3 * qkv_out->d)) return false;
   tc::QkvOut qo = qkv_out ? *qkv_out : tc::QkvOut{};
   qo.packed_kb = Wp ? K / tc::BK : 0;

@@ -8,6 +8,11 @@ from oracle import skipdecode_oracle as O
 from paper_2307_02628_b200 import synth
 
 TOL = {"fp32": 1e-4, "bf16": 3e-2}     # max-abs logit error allowed per storage type
+# Two GPU runs of the same products in bf16 storage that add their fp32 partial sums in a different order
+# (atomic adds in arrival order, another K split, another attention split) differ in the last bits of those
+# sums; where such a sum is then rounded into the bf16 cache or an fp16 operand, a value near a rounding
+# boundary can land on either side, which moves a logit by up to a few 1e-3 at the tested sizes (2.1e-3 seen).
+REORDER_TOL = 5e-3
 
 
 def make_decoder(wl: synth.Workload, weights, full_capacity=False, **kw):

@@ -284,7 +284,7 @@ def test_persistent_gemm_in_the_prompt_pass(B, P):
         err, strict, near = harness.compare(runs[persistent], ref, harness.TOL["bf16"])
         print(f"persistent={persistent} B={B} P={P}: max|err|={err:.3e} argmax strict={strict:.4f} near={near:.4f}")
         assert err <= harness.TOL["bf16"] and near >= 0.99
-    assert float((runs[1] - runs[0]).abs().max()) <= 2e-3     # same products; the residual adds arrive in another order
+    assert float((runs[1] - runs[0]).abs().max()) <= harness.REORDER_TOL     # same products; the residual adds arrive in another order
 
 
 def test_persistent_gemm_with_96_token_tiles():
@@ -307,8 +307,8 @@ def test_persistent_gemm_with_96_token_tiles():
         err, strict, near = harness.compare(runs[mode], ref, harness.TOL["bf16"])
         print(f"persistent={mode}: max|err|={err:.3e} argmax strict={strict:.4f} near={near:.4f}")
         assert err <= harness.TOL["bf16"] and near >= 0.99
-    assert float((runs[1] - runs[2]).abs().max()) <= 2e-3
-    assert float((runs[1] - runs[0]).abs().max()) <= 2e-3
+    assert float((runs[1] - runs[2]).abs().max()) <= harness.REORDER_TOL
+    assert float((runs[1] - runs[0]).abs().max()) <= harness.REORDER_TOL
 
 
 @pytest.mark.parametrize("d,heads,B", [(1024, 8, 20), (1024, 8, 64), (1536, 12, 33), (1536, 12, 100)])
@@ -334,8 +334,8 @@ def test_split_k_under_nonlinear_epilogues(d, heads, B):
             err, strict, near = harness.compare(runs[splitk, graphs], ref, harness.TOL["bf16"])
             print(f"splitk={splitk} graphs={graphs} d={d} B={B}: max|err|={err:.3e} argmax strict={strict:.4f} near={near:.4f}")
             assert err <= harness.TOL["bf16"] and near >= 0.99
-    assert float((runs[8, 1] - runs[0, 1]).abs().max()) <= 2e-3     # same products, partial sums added in another order
-    assert float((runs[8, 1] - runs[8, 0]).abs().max()) <= 2e-3
+    assert float((runs[8, 1] - runs[0, 1]).abs().max()) <= harness.REORDER_TOL     # same products, partial sums added in another order
+    assert float((runs[8, 1] - runs[8, 0]).abs().max()) <= harness.REORDER_TOL
 
 
 @pytest.mark.parametrize("alpha", [2, 3])
@@ -400,7 +400,7 @@ def test_deterministic_option_gives_the_same_bits_every_run(B):
         dec.close()
         _check(runs[-1], ref, "bf16", f"deterministic={det} graphs={graphs} B={B}")
     assert torch.equal(runs[0], runs[1]) and torch.equal(runs[0], runs[2])
-    assert float((runs[0] - runs[3]).abs().max()) <= 2e-3
+    assert float((runs[0] - runs[3]).abs().max()) <= harness.REORDER_TOL
 
 
 def test_expired_device_wait_is_reported_and_the_handle_stays_usable():
@@ -427,4 +427,4 @@ def test_expired_device_wait_is_reported_and_the_handle_stays_usable():
     err, strict, near = harness.compare(again, ref, harness.TOL["bf16"])
     print(f"after an expired wait: max|err|={err:.3e} argmax strict={strict:.4f} with near-ties={near:.4f}")
     assert err <= harness.TOL["bf16"] and near >= 0.99              # 30 (row, step) pairs: one near-tie moves `strict` by 3 %
-    assert float((again - good).abs().max()) <= 2e-3
+    assert float((again - good).abs().max()) <= harness.REORDER_TOL

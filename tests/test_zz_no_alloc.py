@@ -5,7 +5,7 @@ that owns all device memory, or in a serving loop that must not allocate after s
 (the split-KV attention partials) sits in an array inside the library image.  This test
 calls it through the C ABI on two consecutive decode steps and checks each against
 sd_decode_step on the same inputs (the two run the same kernels, so they may differ only by the
-order in which split sums arrive: 2e-3 in bf16 storage, 1e-5 in fp32) and against the CPU oracle
+order in which split sums arrive: 5e-3 in bf16 storage, 1e-5 in fp32) and against the CPU oracle
 with the tolerance of the other parity tests.
 
 It is collected last on purpose: if it fails, a run that stops at the first failure has
@@ -32,7 +32,7 @@ def test_static_scratch_step_matches_regular_step_twice_in_a_row(name, shape):
     dec = harness.make_decoder(wl, w)
     dec.set_option(binding.SD_OPT_ATTN_CHUNK, 32)          # several splits per (row, head): the scratch is really used
     tol = harness.TOL[name]
-    same = {"fp32": 1e-5, "bf16": 2e-3}[name]               # one GPU path against the other
+    same = {"fp32": 1e-5, "bf16": harness.REORDER_TOL}[name]               # one GPU path against the other
     ref = harness.oracle_run_forced(wl, w, prompts, forced)    # [B, 1 + gen_len, vocab], index 0 = prompt pass
     with torch.cuda.stream(dec.stream):
         dec.schedule(wl.max_layers, wl.min_layers, wl.warmup, wl.gen_len)
