@@ -233,6 +233,8 @@ def measure_workload(name, wl, weights, args, device, dist, world, steps, warmup
         dec.set_option(binding.SD_OPT_PDL, args.pdl)
     if args.deterministic:
         dec.set_option(binding.SD_OPT_DETERMINISTIC, 1)
+    if args.attn_staged is not None:
+        dec.set_option(binding.SD_OPT_ATTN_STAGED, args.attn_staged)
     if args.attn_chunk:
         dec.set_option(binding.SD_OPT_ATTN_CHUNK, args.attn_chunk)
     prompts = synth.make_prompts(wl).to(device)
@@ -477,6 +479,7 @@ def main():
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")
     ap.add_argument("--deterministic", action="store_true", help="SD_OPT_DETERMINISTIC = 1")
+    ap.add_argument("--attn-staged", type=int, default=None, help="SD_OPT_ATTN_STAGED: 0 = register-only decode attention everywhere")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true", help="with the default workload (c4): do not also time c3 and c5")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -279,11 +279,15 @@ enum {
                               can differ in the last bits; 1: these products park their partial tiles like the others and
                               the block that arrives last adds them in split order: every run gives the same bits,
                               at a tenth to a fifth of the decode rate (a second pass over every tile of those products) */
-  SD_OPT_TEST_WAIT_EXPIRY = 13 /* test hook, one shot: the next tensor-core product never reports its accumulator
+  SD_OPT_TEST_WAIT_EXPIRY = 13, /* test hook, one shot: the next tensor-core product never reports its accumulator
                               complete, its epilogue gives up the bounded wait after about a millisecond, writes
                               nothing, and sets the wait-expired bit of the status word (sd_status then returns
                               SD_ERR_DEVICE).  Nothing is left in flight and the handle stays usable: the following
                               sd_prefill clears the status word.  The step that contained the product returns garbage. */
+  SD_OPT_ATTN_STAGED = 14    /* bf16 storage: 1 (default) = decode-attention launches with at least 12 (row, head) pairs per
+                              SM stream K and V through a ring of shared-memory stages filled by 8 KB bulk copies;
+                              0 = every launch uses the kernel that loads them straight into registers (as fp32 storage
+                              and smaller launches always do) */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff

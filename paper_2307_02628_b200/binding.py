@@ -17,7 +17,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libskipdec
 _lib = None
 
 SD_OK, SD_ERR_ARG, SD_ERR_STATE, SD_ERR_POSITION, SD_ERR_CAPACITY, SD_ERR_CUDA, SD_ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
-SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING, SD_OPT_PDL, SD_OPT_PREFILL_ATTN, SD_OPT_GEMM_PERSISTENT, SD_OPT_GEMM_SPLITK, SD_OPT_DETERMINISTIC, SD_OPT_TEST_WAIT_EXPIRY = 1, 2, 3, 4, 5, 8, 10, 11, 12, 13
+SD_OPT_GRAPHS, SD_OPT_ATTN_CHUNK, SD_OPT_GEMM, SD_OPT_TIMING, SD_OPT_PDL, SD_OPT_PREFILL_ATTN, SD_OPT_GEMM_PERSISTENT, SD_OPT_GEMM_SPLITK, SD_OPT_DETERMINISTIC, SD_OPT_TEST_WAIT_EXPIRY, SD_OPT_ATTN_STAGED = 1, 2, 3, 4, 5, 8, 10, 11, 12, 13, 14
 KERNEL_CLASSES = ("embed", "layernorm", "gemm_qkv", "kv_append", "attention", "lm_head", "gemm_out", "gemm_fc1", "gemm_fc2")
 
 EXPORTS = ("sd_arena_bytes", "sd_create", "sd_schedule", "sd_schedule_compute", "sd_schedule_power_compute",

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libskipdecode.so")
 SOURCES = [os.path.join(CSRC, "skipdecode.cu")]
-HEADERS = [os.path.join(CSRC, n) for n in ("kernels.cuh", "gemm_tc.cuh", "sample.cuh", "attn_prefill.cuh", "gemm_persist.cuh")] + \
+HEADERS = [os.path.join(CSRC, n) for n in ("kernels.cuh", "gemm_tc.cuh", "sample.cuh", "attn_prefill.cuh", "gemm_persist.cuh", "attn_stream.cuh")] + \
           [os.path.join(os.path.dirname(PKG), "include", "skipdecode.h")]
 
 

@@ -18,6 +18,7 @@
 #include "gemm_persist.cuh"
 #include "sample.cuh"
 #include "attn_prefill.cuh"
+#include "attn_stream.cuh"
 
 namespace {
 
@@ -68,6 +69,8 @@ struct sd_handle {
   int64_t steps = 0, layer_steps = 0, launches = 0;
   // options
   int opt_graphs = 1, opt_chunk = 0, opt_gemm = 0, opt_timing = 0, opt_pdl = SD_PDL_DEFAULT, opt_prefill = 1;
+  int opt_attn_staged = 1;   // decode attention in bf16 storage through the shared-memory ring where that pays; 0: never
+  unsigned attn_stream_ready = 0;   // bit per head size whose shared-memory attributes are set
   bool packed = false;       // the arena holds tile-packed copies of the weight matrices
   // graphs: key = (B, n, warmup, chunk, n_chunks, ids ptr, logits ptr)
   struct Graph { cudaGraphExec_t exec; int64_t nodes; };
@@ -190,7 +193,8 @@ void carve(const sd_config& c, const sd_plan& p, Arena& A) {
   A.part_slots = std::max((size_t)c.max_batch * H * ((maxT + kMinChunk - 1) / kMinChunk), R * H);
   A.part_acc = take(A.part_slots * hd * 4);
   A.part_ml = take(A.part_slots * 2 * 4);
-  A.counters = take(R * H * 4);          // split-KV arrival counters, one per (row, head); zero between launches
+  A.counters = take((R * H + 64) * 4);   // split-KV arrival counters, one per (row, head), then the persistent attention
+                                         // kernel's work counter; all zero between launches
   A.row_index = take((size_t)c.max_batch * 4);
   A.ids = take((size_t)c.max_batch * 4);
   A.logits = take((size_t)c.max_batch * c.vocab * 4);
@@ -291,10 +295,47 @@ bool launch_qkv_to_cache<bf16>(Launcher& Lc, const bf16* u, const bf16* W, size_
   return done;
 }
 
+// Decode attention with K and V staged through shared memory (bf16 storage).  Returns false when the
+// kernel cannot be prepared; the register-only kernel then takes the launch.
+template <int HD>
+bool launch_attention_stream(Launcher& Lc, const bf16* Kc, const bf16* Vc, int cap, int rows, sd::RowMap map, int chunk, int n_chunks) {
+  sd_handle* h = Lc.h;
+  constexpr int smem = sd::as::smem_bytes();
+  const unsigned bit = HD == 128 ? 1u : HD == 64 ? 2u : 4u;
+  if (!(h->attn_stream_ready & bit)) {       // per handle: the attributes belong to the handle's device
+    if (cudaFuncSetAttribute(sd::attn_stream_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(sd::attn_stream_kernel<HD>, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    h->attn_stream_ready |= bit;
+  }
+  const int H = h->cfg.n_heads;
+  Lc.begin(SD_K_ATTENTION);
+  dim3 grid(rows * H, n_chunks);
+  sd::launch_kernel(pdl_for(h, SD_K_ATTENTION), h->stream, sd::attn_stream_kernel<HD>, dim3(grid), dim3(sd::as::THREADS), smem,
+                    (const float*)h->at<float>(h->A.qkv), 3 * h->cfg.d_model, Kc, Vc, cap, H, map, chunk, n_chunks, Lc.part_acc, Lc.part_ml,
+                    h->at<int>(h->A.counters), h->at<bf16>(h->A.o), h->status());
+  Lc.end();
+  return true;
+}
+
+// Which decode-attention kernel takes a launch of rows x H (row, head) pairs in bf16 storage.  The staged kernel
+// holds 3 blocks per SM, the register-only one 7: the staged one pays where the launch is many times its
+// 3 x SMs slots (config 4: 2048 pairs, +1.6 % tokens/s; config 5: 8192, +0.6 %), and loses where the other holds
+// the whole launch in one wave (config 3: 1024 pairs, -12 %).
+bool attn_staged(const sd_handle* h, int rows) {
+  return h->cfg.dtype == SD_DTYPE_BF16 && h->opt_attn_staged &&
+         (long)rows * h->cfg.n_heads >= 4L * sd::as::BLOCKS_PER_SM * h->tc.sm_count;
+}
+
 template <typename T, int HD>
 void launch_attention_hd(Launcher& Lc, const T* Kc, const T* Vc, int cap, int rows, sd::RowMap map, int chunk,
                          int n_chunks) {
   sd_handle* h = Lc.h;
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (attn_staged(h, rows) && launch_attention_stream<HD>(Lc, Kc, Vc, cap, rows, map, chunk, n_chunks)) return;
+  }
   const int H = h->cfg.n_heads;
   Lc.begin(SD_K_ATTENTION);
   dim3 grid(rows * H, n_chunks);
@@ -409,7 +450,8 @@ void enqueue_head(Launcher& Lc, int rows, const int* row_index, float* d_logits)
 int pick_chunk(const sd_handle* h, int rows, int T) {
   if (h->opt_chunk > 0) return h->opt_chunk;
   const long rh = (long)rows * h->cfg.n_heads;
-  const long slots = 7L * h->tc.sm_count;           // blocks resident at once (7 per SM by registers)
+  // blocks resident at once: 7 per SM by registers for the register-only kernel, 3 rings per SM for the staged one
+  const long slots = (attn_staged(h, rows) ? (long)sd::as::BLOCKS_PER_SM : 7L) * h->tc.sm_count;
   const int whole = (h->cfg.max_prompt + h->cfg.max_gen + kMinChunk - 1) / kMinChunk * kMinChunk;
   int best = whole;
   double best_cost = 1e30;
@@ -583,7 +625,7 @@ int sd_create(const sd_config* cfg, const sd_weights* w, const sd_plan* plan, vo
   h->arena = static_cast<char*>(arena);
   h->stream = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(h->arena + h->A.scalars, 0, 256, h->stream) != cudaSuccess ||
-      cudaMemsetAsync(h->arena + h->A.counters, 0, (size_t)h->A.rows_max * cfg->n_heads * 4, h->stream) != cudaSuccess) {
+      cudaMemsetAsync(h->arena + h->A.counters, 0, ((size_t)h->A.rows_max * cfg->n_heads + 64) * 4, h->stream) != cudaSuccess) {
     cudaGetLastError(); delete h; return SD_ERR_CUDA;
   }
   if (cfg->dtype == SD_DTYPE_BF16) {
@@ -704,7 +746,11 @@ int sd_prefill(sd_handle* h, const int32_t* d_tokens, int B, int P, float* d_log
   }
   if (h->have_rows) { h->have_rows = false; h->rows.clear(); drop_graphs(h); }   // a new batch: all rows generate
   // a new batch starts with a clean status word (a bit set earlier has been reported through sd_status by now or is lost)
-  if (cudaMemsetAsync(h->status(), 0, sizeof(int), h->stream) != cudaSuccess) { cudaGetLastError(); return SD_ERR_CUDA; }
+  if (cudaMemsetAsync(h->status(), 0, sizeof(int), h->stream) != cudaSuccess ||
+      cudaMemsetAsync(h->arena + h->A.counters, 0, ((size_t)h->A.rows_max * h->cfg.n_heads + 64) * 4, h->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return SD_ERR_CUDA;
+  }
   const int err = h->cfg.dtype == SD_DTYPE_BF16 ? run_prefill<bf16>(h, d_tokens, B, P, d_logits)
                                                 : run_prefill<float>(h, d_tokens, B, P, d_logits);
   if (err) return err;
@@ -886,6 +932,9 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value < 0 || value >= (1 << SD_K_COUNT)) return SD_ERR_ARG;
       if (value != h->opt_pdl) drop_graphs(h);
       h->opt_pdl = value; return SD_OK;
+    case SD_OPT_ATTN_STAGED:
+      if ((value != 0) != (h->opt_attn_staged != 0)) drop_graphs(h);
+      h->opt_attn_staged = value ? 1 : 0; return SD_OK;
     case SD_OPT_DETERMINISTIC:
       if ((value != 0) != (h->tc.deterministic != 0)) drop_graphs(h);
       h->tc.deterministic = value ? 1 : 0; return SD_OK;
