@@ -74,6 +74,14 @@ def step_bytes(wl: synth.Workload, n_active) -> float:
 # taken on: the hash below is checked and `traffic` is null once the kernel text has changed.
 ATTN_TRAFFIC_RATIO = 1.0057
 ATTN_KERNEL_SHA256 = "31a94a145b5ed8ac87c0b55544c26e415ec060262f217260c54eeee81869bd3d"
+# attn_stream_kernel (the staged kernel, which takes the launches of at least 12 (row, head) pairs per SM): DRAM bytes
+# beyond K and V per launch, from ncu --set full captures at two launch shapes, keyed by (d_model, heads, batch).
+# Config 4's shape at T = 1027: 1.077985 GB read + 4.18 MB written for 1.076888 GB of K and V; config 5's at T = 259:
+# 1.090583 GB + 5.55 MB for 1.086324 GB.  The surplus is q, the output rows and the sectors at the ends of the
+# streams, none of which grows with T, so it is added per launch rather than as a factor.  Valid for the kernel source
+# the captures were taken on (hash of attn_stream.cuh).
+ATTN_STREAM_EXTRA_BYTES = {(4096, 32, 64): 5.27e6, (4096, 32, 256): 9.81e6}
+ATTN_STREAM_SHA256 = "a2197a93fa28a4e060c0c5f931e3017c1017dc356643d126225f2708029b22c9"
 
 
 def attention_kernel_hash() -> str:
@@ -82,6 +90,17 @@ def attention_kernel_hash() -> str:
     i = src.index("template <typename T, int HD, int UNROLL>")
     j = src.index("// Host side: launch with the programmatic")
     return hashlib.sha256(src[i:j].encode()).hexdigest()
+
+
+def staged_kernel_hash() -> str:
+    import hashlib
+    return hashlib.sha256(open(os.path.join(ROOT, "paper_2307_02628_b200", "csrc", "attn_stream.cuh")).read().encode()).hexdigest()
+
+
+def uses_staged_attention(wl, args) -> bool:
+    """The library's rule (skipdecode.cu, attn_staged): bf16 storage and at least 12 (row, head) pairs per SM."""
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    return wl.shape.dtype == "bf16" and args.attn_staged != 0 and wl.batch * wl.shape.n_heads >= 12 * sms
 
 
 # --------------------------------------------------------------------------- ranks
@@ -372,20 +391,31 @@ def measure_workload(name, wl, weights, args, device, dist, world, steps, warmup
     dec.close()
     torch.cuda.empty_cache()
     return {"name": name, "wl": wl, "G_run": G_run, "n_active": n_active, "ms_step": ms_step, "launches": launches,
+            "staged": uses_staged_attention(wl, args),
             "clocks": clock_info, "e2e_s": e2e_s, "attn_bytes": attn_bytes, "kt": kt, "full": full, "prefill_s": t_prefill}
 
 
 def roofline_entry(r, peak, peak_kind):
     """The dominant kernel's roofline object from a measure_workload result."""
-    s = r["wl"].shape
+    wl = r["wl"]
+    s = wl.shape
     attn_ms, attn_n = r["kt"]["attention"]
     achieved = r["attn_bytes"] / (attn_ms / 1e3) / 1e9 if attn_ms > 0 else None
-    same_kernel = attention_kernel_hash() == ATTN_KERNEL_SHA256 and s.dtype == "bf16"
-    return {"kernel": "attn_partial_kernel (split-KV decode attention)", "bound": "hbm", "achieved": achieved,
+    traffic = source = None
+    if r["staged"]:
+        kernel = "attn_stream_kernel (split-KV decode attention, K and V staged through shared memory by bulk copies)"
+        extra = ATTN_STREAM_EXTRA_BYTES.get((s.d_model, s.n_heads, wl.batch))
+        if attn_n and extra is not None and staged_kernel_hash() == ATTN_STREAM_SHA256:
+            traffic = r["attn_bytes"] / attn_n + extra
+            source = "K and V bytes of a launch + the surplus an ncu capture of this kernel source measured at this launch shape on a 2-layer case"
+    else:
+        kernel = "attn_partial_kernel (split-KV decode attention)"
+        if attn_n and s.dtype == "bf16" and attention_kernel_hash() == ATTN_KERNEL_SHA256:
+            traffic = ATTN_TRAFFIC_RATIO * r["attn_bytes"] / attn_n
+            source = "ncu capture of this kernel source on a 2-layer case of config 4's launch shape, scaled by the keys read"
+    return {"kernel": kernel, "bound": "hbm", "achieved": achieved,
             "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
-            "traffic": (ATTN_TRAFFIC_RATIO * r["attn_bytes"] / attn_n if attn_n and same_kernel else None),
-            "traffic_source": ("ncu capture of this kernel source on a 2-layer case of the same launch shape, scaled by the keys read"
-                               if attn_n and same_kernel else None),
+            "traffic": traffic, "traffic_source": source,
             "launches_timed": int(attn_n),
             "algorithmic_bytes_per_launch": r["attn_bytes"] / attn_n if attn_n else None}
 
