@@ -180,11 +180,11 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
           kv_base = n < 2 * qo.d ? qo.Kc : qo.Vc;
         }
       }
+      const float b = (bias != nullptr && n < N) ? __bfloat162float(bias[n]) : 0.f;   // a weight: fetched before the wait
       ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, status);
       if (tile + (int)gridDim.x >= tiles_total) pdl_launch_dependents();   // this CTA's last main loop is over
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const float b = (bias != nullptr && n < N) ? __bfloat162float(bias[n]) : 0.f;
 #pragma unroll 1
       for (int c = 0; c < NB; c += 32) {
         uint32_t r[32];

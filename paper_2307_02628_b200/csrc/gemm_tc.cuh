@@ -300,6 +300,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         kv_base = n < 2 * qo.d ? qo.Kc : qo.Vc;
       }
     }
+    // the bias is a weight: fetched now, so that its latency hides behind the main loop.  It goes in once: with the
+    // fix-up by the block that finishes the tile, else by the first split
+    const bool fix = (EPI != EPI_RESIDUAL_F32 || qo.fix_residual) && gridDim.z > 1;
+    const float b = (bias != nullptr && n < N && (fix || EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
     const bool accum_ok = mbar_wait(accum_bar, 0, abort_flag, status, qo.test_expire ? 2000000LL : kWaitLimit);
     // The main loop is over: let the next kernel of the stream become resident now, so that its
     // launch and set-up overlap this kernel's epilogue (earlier would only park its blocks on the
@@ -307,7 +311,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     pdl_launch_dependents();
     // K split under a non-linear epilogue: park the partial tile, count arrivals, and let
     // the block that arrives last finish the tile from the parked partials
-    const bool fix = (EPI != EPI_RESIDUAL_F32 || qo.fix_residual) && gridDim.z > 1;
     bool go = accum_ok;
     if (fix) {
       // the fix-up meets at a named barrier: all epilogue threads take it or none (a bounded wait may
@@ -319,8 +322,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
     if (go) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // the bias goes in once: with the fix-up by the block that finishes the tile, else by the first split
-      const float b = (bias != nullptr && n < N && (fix || EPI != EPI_RESIDUAL_F32 || blockIdx.z == 0)) ? __bfloat162float(bias[n]) : 0.f;
       const int c_begin = ((warp - 2) >> 2) * GROUP_COLS;
       const int splits = (int)gridDim.z, tile_id = (int)(blockIdx.y * gridDim.x + blockIdx.x);
       float* ws_tile = fix ? qo.ws + (size_t)tile_id * splits * (NB * BM) + quarter * 32 + lane : nullptr;
