@@ -291,10 +291,12 @@ enum {
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff
-/* Default: the five GEMM classes.  A GEMM that starts early sets up its barriers and tensor
- * memory and streams its first weight tiles while its predecessor drains (measured +1.5 % at the
- * OPT-6.7B shape); starting the attention kernel or the LayerNorms early costs 2-5 %. */
-#define SD_PDL_DEFAULT ((1 << 2) | (1 << 5) | (1 << 6) | (1 << 7) | (1 << 8))
+/* Default: the five GEMM classes and the LayerNorms.  A GEMM that starts early sets up its barriers and
+ * tensor memory and streams its first weight tiles while its predecessor drains (measured +1.5 % at the
+ * OPT-6.7B shape); a LayerNorm that starts early saves its launch latency after the residual product, which is
+ * nothing at the OPT-6.7B shape and +3 % / +5 % at the OPT-1.3B / OPT-125M shapes, where the products are short;
+ * starting the attention kernel early gains nothing anywhere and costs 7 % at the OPT-1.3B shape. */
+#define SD_PDL_DEFAULT ((1 << 1) | (1 << 2) | (1 << 5) | (1 << 6) | (1 << 7) | (1 << 8))
 
 /* Device time and launch count accumulated per kernel class while SD_OPT_TIMING is
  * on; synchronises the stream.  ms, launches: host. */
