@@ -428,3 +428,20 @@ def test_expired_device_wait_is_reported_and_the_handle_stays_usable():
     print(f"after an expired wait: max|err|={err:.3e} argmax strict={strict:.4f} with near-ties={near:.4f}")
     assert err <= harness.TOL["bf16"] and near >= 0.99              # 30 (row, step) pairs: one near-tie moves `strict` by 3 %
     assert float((again - good).abs().max()) <= harness.REORDER_TOL
+
+
+def test_weight_beyond_the_fp16_range_is_reported_at_create():
+    # bf16 storage multiplies fp16 copies of the weights: a weight above 65504 is clipped in the copy and bit 8 of the
+    # status word says so right after sd_create; weights inside the range leave the word at zero
+    from paper_2307_02628_b200 import binding
+    shape = synth.ModelShape("range-bf16", 1, 256, 4, 512, 640, 64, "bf16")
+    wl = synth.Workload(shape, 2, 8, 2, 1, 1, 0)
+    w = synth.make_weights(shape, seed=3)
+    dec = harness.make_decoder(wl, w)
+    assert dec.status() == 0
+    dec.close()
+    w["layers"][0]["w_fc1"][5, 7] = 1.0e5
+    dec = harness.make_decoder(wl, w)
+    assert dec.status() == 8
+    dec.close()
+

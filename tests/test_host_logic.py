@@ -111,3 +111,24 @@ def test_power_law_schedule_rejects_what_its_integers_cannot_hold():
     # well inside the limit the table is still the oracle's
     assert binding.schedule_power_compute(32, 32, 4, 0, 4097, 8) == tuple(O.schedule_power(32, 4, 0, 4097, 32, 8))
     assert binding.schedule_power_compute(32, 32, 4, 0, 65536, 4) == tuple(O.schedule_power(32, 4, 0, 65536, 32, 4))
+
+
+def test_bf16_weights_are_fp16_values_inside_the_fp16_range():
+    # What the packed weight copies rely on: a bf16 has 8 significant bits, an fp16 has 11, so every bf16 whose
+    # magnitude lies in [2^-14, 65504] is an fp16 value exactly; below that it lands on the fp16 subnormal grid
+    # (spacing 2^-24, error at most 2^-25); above it the conversion has to clip.  All 65 536 bit patterns.
+    import torch
+    bits = torch.arange(65536, dtype=torch.int32).to(torch.int16)
+    v = bits.view(torch.bfloat16).to(torch.float64)
+    finite = torch.isfinite(v)
+    mag = v.abs()
+    normal = finite & (mag >= 2.0 ** -14) & (mag <= 65504.0)
+    as_f16 = v.to(torch.float16).to(torch.float64)
+    assert int(normal.sum()) == 2 * 30 * 128                # 30 binades, 128 mantissas, two signs
+    assert torch.equal(as_f16[normal], v[normal])
+    small = finite & (mag < 2.0 ** -14)
+    assert float((as_f16[small] - v[small]).abs().max()) <= 2.0 ** -25
+    big = finite & (mag > 65504.0)
+    assert bool(torch.isinf(as_f16[big]).all())              # a plain conversion overflows: the pack kernel saturates instead
+    # the largest bf16 below the limit is exactly representable, the next one is not
+    assert float(v[normal].abs().max()) == 65280.0
