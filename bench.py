@@ -98,9 +98,12 @@ def staged_kernel_hash() -> str:
 
 
 def uses_staged_attention(wl, args) -> bool:
-    """The library's rule (skipdecode.cu, attn_staged): bf16 storage and at least 12 (row, head) pairs per SM."""
+    """The library's rule (skipdecode.cu, attn_staged): bf16 storage, at least 12 (row, head) pairs per SM, and a
+    handle configured for at least 1024 positions (option value 2 drops the last condition)."""
     sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
-    return wl.shape.dtype == "bf16" and args.attn_staged != 0 and wl.batch * wl.shape.n_heads >= 12 * sms
+    if wl.shape.dtype != "bf16" or args.attn_staged == 0 or wl.batch * wl.shape.n_heads < 12 * sms:
+        return False
+    return args.attn_staged == 2 or wl.prompt_len + wl.gen_len >= 1024
 
 
 # --------------------------------------------------------------------------- ranks
@@ -509,7 +512,7 @@ def main():
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")
     ap.add_argument("--deterministic", action="store_true", help="SD_OPT_DETERMINISTIC = 1")
-    ap.add_argument("--attn-staged", type=int, default=None, help="SD_OPT_ATTN_STAGED: 0 = register-only decode attention everywhere")
+    ap.add_argument("--attn-staged", type=int, default=None, help="SD_OPT_ATTN_STAGED: 0 = register-only decode attention everywhere, 2 = staged whatever the sequence length")
     ap.add_argument("--no-full-layer", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true", help="with the default workload (c4): do not also time c3 and c5")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -285,9 +285,10 @@ enum {
                               SD_ERR_DEVICE).  Nothing is left in flight and the handle stays usable: the following
                               sd_prefill clears the status word.  The step that contained the product returns garbage. */
   SD_OPT_ATTN_STAGED = 14    /* bf16 storage: 1 (default) = decode-attention launches with at least 12 (row, head) pairs per
-                              SM stream K and V through a ring of shared-memory stages filled by 8 KB bulk copies;
-                              0 = every launch uses the kernel that loads them straight into registers (as fp32 storage
-                              and smaller launches always do) */
+                              SM, on a handle configured for at least 1024 positions (max_prompt + max_gen), stream K and V
+                              through a ring of shared-memory stages filled by 8 KB bulk copies; 2 = the same without the
+                              length condition; 0 = every launch uses the kernel that loads them straight into registers
+                              (as fp32 storage and smaller launches always do) */
 };
 int sd_set_option(sd_handle *h, int option, int value);
 #define SD_PDL_ALL 0x1ff

@@ -321,12 +321,15 @@ bool launch_attention_stream(Launcher& Lc, const bf16* Kc, const bf16* Vc, int c
 }
 
 // Which decode-attention kernel takes a launch of rows x H (row, head) pairs in bf16 storage.  The staged kernel
-// holds 3 blocks per SM, the register-only one 7: the staged one pays where the launch is many times its
-// 3 x SMs slots (config 4: 2048 pairs, +1.6 % tokens/s; config 5: 8192, +0.6 %), and loses where the other holds
-// the whole launch in one wave (config 3: 1024 pairs, -12 %).
+// holds 3 blocks per SM, the register-only one 7, and a staged block needs a few microseconds before its first keys
+// arrive.  Measured: it pays where the launch is many times its 3 x SMs slots and the rows are long (config 4: 2048
+// pairs, 1025..1536 keys, +1.6 % tokens/s; config 5: 8192 pairs, 257..1280 keys, +0.6 %), is level at 512..1024 keys,
+// loses at 60..160 keys (-2.3 %) and loses where the other kernel holds the whole launch in one wave (config 3: 1024
+// pairs, -12 %).  The length that counts is the handle's maximum, so that the choice does not change inside a sequence.
 bool attn_staged(const sd_handle* h, int rows) {
-  return h->cfg.dtype == SD_DTYPE_BF16 && h->opt_attn_staged &&
-         (long)rows * h->cfg.n_heads >= 4L * sd::as::BLOCKS_PER_SM * h->tc.sm_count;
+  if (h->cfg.dtype != SD_DTYPE_BF16 || !h->opt_attn_staged) return false;
+  if ((long)rows * h->cfg.n_heads < 4L * sd::as::BLOCKS_PER_SM * h->tc.sm_count) return false;
+  return h->opt_attn_staged == 2 || h->cfg.max_prompt + h->cfg.max_gen >= 1024;
 }
 
 template <typename T, int HD>
@@ -933,8 +936,9 @@ int sd_set_option(sd_handle* h, int option, int value) {
       if (value != h->opt_pdl) drop_graphs(h);
       h->opt_pdl = value; return SD_OK;
     case SD_OPT_ATTN_STAGED:
-      if ((value != 0) != (h->opt_attn_staged != 0)) drop_graphs(h);
-      h->opt_attn_staged = value ? 1 : 0; return SD_OK;
+      if (value != h->opt_attn_staged) drop_graphs(h);
+      if (value < 0 || value > 2) return SD_ERR_ARG;
+      h->opt_attn_staged = value; return SD_OK;
     case SD_OPT_DETERMINISTIC:
       if ((value != 0) != (h->tc.deterministic != 0)) drop_graphs(h);
       h->tc.deterministic = value ? 1 : 0; return SD_OK;

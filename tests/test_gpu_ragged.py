@@ -10,7 +10,7 @@ from paper_2307_02628_b200 import binding, synth
 pytestmark = pytest.mark.gpu
 
 
-def _run(shape, B, P, G, mx, mn, warm, pad, retire, graphs=1, tiles=1, seed=12):
+def _run(shape, B, P, G, mx, mn, warm, pad, retire, graphs=1, tiles=1, seed=12, options=None):
     """retire: {step g: rows that generate from step g on}.  Returns the worst logit error."""
     wl = synth.Workload(shape, B, P, G, mx, mn, warm)
     w = synth.make_weights(shape, seed=seed, random_ln=True)
@@ -21,6 +21,8 @@ def _run(shape, B, P, G, mx, mn, warm, pad, retire, graphs=1, tiles=1, seed=12):
     dec = harness.make_decoder(wl, w)
     dec.set_option(binding.SD_OPT_GRAPHS, graphs)
     dec.set_option(binding.SD_OPT_PREFILL_ATTN, tiles)
+    for opt, value in (options or {}).items():
+        dec.set_option(opt, value)
     worst = 0.0
     agree = total = 0
     with torch.cuda.stream(dec.stream):
