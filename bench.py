@@ -249,6 +249,8 @@ def measure_workload(name, wl, weights, args, device, dist, world, steps, warmup
         dec.set_option(binding.SD_OPT_GEMM, args.gemm_mode)
     if args.no_persistent:
         dec.set_option(binding.SD_OPT_GEMM_PERSISTENT, 0)
+    elif args.persistent_tiles is not None:
+        dec.set_option(binding.SD_OPT_GEMM_PERSISTENT, args.persistent_tiles)
     if args.splitk is not None:
         dec.set_option(binding.SD_OPT_GEMM_SPLITK, args.splitk)
     if args.pdl is not None:
@@ -508,6 +510,7 @@ def main():
     ap.add_argument("--select", default="greedy", choices=["greedy", "top-p"],
                     help="token selection in the timed generation loop (the five configurations are greedy)")
     ap.add_argument("--no-persistent", action="store_true", help="SD_OPT_GEMM_PERSISTENT = 0")
+    ap.add_argument("--persistent-tiles", type=int, default=None, help="SD_OPT_GEMM_PERSISTENT: 1 = 96- or 128-token tiles (default), 2 = 128 only")
     ap.add_argument("--splitk", type=int, default=None, help="SD_OPT_GEMM_SPLITK (most splits of K under a non-linear epilogue; 0 = off)")
     ap.add_argument("--attn-chunk", type=int, default=0, help="SD_OPT_ATTN_CHUNK (0 automatic)")
     ap.add_argument("--pdl", type=int, default=None, help="SD_OPT_PDL mask of kernel classes (0 = off)")
