@@ -17,6 +17,24 @@ def test_library_exports_every_declared_symbol(repo_root):
         assert hasattr(L, name), name
 
 
+def test_binding_constants_are_the_headers(repo_root):
+    # the ctypes binding restates the header's enumerators: option numbers, error codes, kernel classes
+    hdr = open(os.path.join(repo_root, "include", "skipdecode.h")).read()
+    enums = {name: int(value, 0) for name, value in re.findall(r"\b(SD_[A-Z0-9_]+)\s*=\s*(-?(?:0x[0-9a-fA-F]+|\d+))", hdr)}
+    checked = 0
+    for name, value in enums.items():
+        if hasattr(binding, name):
+            assert getattr(binding, name) == value, name
+            checked += 1
+    assert checked >= 15
+    for name in ("SD_OPT_GRAPHS", "SD_OPT_ATTN_CHUNK", "SD_OPT_GEMM", "SD_OPT_TIMING", "SD_OPT_PDL", "SD_OPT_PREFILL_ATTN",
+                 "SD_OPT_GEMM_PERSISTENT", "SD_OPT_GEMM_SPLITK", "SD_OPT_DETERMINISTIC", "SD_OPT_TEST_WAIT_EXPIRY",
+                 "SD_OPT_ATTN_STAGED"):
+        assert name in enums and hasattr(binding, name), name
+    classes = [n for n in enums if n.startswith("SD_K_") and n != "SD_K_COUNT"]
+    assert enums["SD_K_COUNT"] == len(classes) == len(binding.KERNEL_CLASSES)
+
+
 SCHEDULES = [(4, 4, 2, 0, 32), (12, 12, 4, 0, 128), (24, 24, 8, 0, 256), (32, 32, 8, 0, 512), (32, 32, 4, 0, 1024),
              (32, 22, 11, 1, 1024), (32, 14, 8, 1, 512), (32, 10, 6, 1, 100), (32, 8, 5, 1, 1024),
              (24, 16, 8, 1, 512), (24, 10, 6, 1, 100), (24, 7, 5, 1, 37), (24, 6, 4, 1, 3),
